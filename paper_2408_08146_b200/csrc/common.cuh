@@ -1,0 +1,165 @@
+// Shared device helpers and the internal launcher interface of libkoala.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+typedef __nv_bfloat16 bf16;
+
+namespace koala {
+
+// ---------------------------------------------------------------------------------------------
+// scalar conversions
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// Programmatic dependent launch: every kernel lets its successor start early and waits for its
+// predecessor before touching anything the predecessor may have written.  Both are no-ops when
+// the launch did not opt in.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// A matrix given as the sum of `n` partial matrices `stride` floats apart (split-K results).
+struct SplitIn {
+  const float *p;
+  int n;
+  size_t stride;
+  int ld;
+  __device__ __forceinline__ float at(int r, int c) const {
+    const float *q = p + (size_t)r * ld + c;
+    float v = q[0];
+    for (int s = 1; s < n; ++s) v += q[(size_t)s * stride];
+    return v;
+  }
+};
+
+// Per-row plan of one forward over R rows (rows_per_seq consecutive rows per sequence).
+struct RowPlan {
+  const int32_t *pos;     // [R] RoPE position
+  const int32_t *slot;    // [R] KV slot to write, -1 = row not in use
+  const uint64_t *mask;   // [R][2] visibility over the slots ctx_len .. ctx_len+127
+  const int32_t *ctx_len; // [B] slots 0..ctx_len-1 are visible to every row of the sequence
+  const int32_t *kv_len;  // [B] slots in use after this forward's writes
+  const float2 *rope;     // [R][head_dim/2] (cos, sin)
+};
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                   cudaStream_t stream, bool pdl, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
+// ---------------------------------------------------------------------------------------------
+// launcher interface (one per kernel family); every launcher is asynchronous on `st`
+// ---------------------------------------------------------------------------------------------
+struct Launch {
+  cudaStream_t st;
+  bool pdl;
+};
+
+struct GemmMats {         // up to three weight matrices sharing K_in, outputs concatenated
+  const void *W[3];
+  int n_out[3];
+  int n;
+};
+
+// ops.cu
+cudaError_t embed_norm(Launch L, int dtype, const int32_t *tok, const void *E, const void *g,
+                       float *x, void *xn, int R, int H, int V, float eps);
+// mode 0: v = x + sum(P); 1: v = sum(P) + bias; 2: v = x + SiLU(sum(P) + bias).  x <- v;
+// n = g ? rmsnorm(v) * g : v;  xn <- T(n) if xn;  out_f32 <- n if out_f32.
+cudaError_t row_epilogue(Launch L, int dtype, int mode, float *x, SplitIn P, const void *bias,
+                         const void *g, void *xn, float *out_f32, int R, int H, float eps);
+cudaError_t eagle_concat(Launch L, int dtype, const float *feat_src, const int32_t *row_src,
+                         const int32_t *row_tok, const void *E, void *cat, int R, int H, int V);
+cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowPlan plan, float *q_out,
+                          void *k_cache, void *v_cache, int R, int rows_per_seq, int n_heads,
+                          int head_dim, int S_max);
+cudaError_t swiglu(Launch L, int dtype, SplitIn gu, void *act, int R, int F);
+cudaError_t tree_attention(Launch L, int dtype, const float *q, const void *k_cache,
+                           const void *v_cache, RowPlan plan, void *out, int R, int rows_per_seq,
+                           int B, int n_heads, int head_dim, int S_max);
+cudaError_t argmax_rows(Launch L, const float *logits, int32_t *out, int R, int V);
+cudaError_t topk_logp(Launch L, const float *logits, int32_t *tok, float *logp, int R, int V, int k);
+// dst[r] = T(src[row_src ? row_src[r] : r]); optionally dst32[r * dst32_stride] = the same row in fp32
+cudaError_t cast_rows(Launch L, int dtype, const float *src, const int32_t *row_src, void *dst,
+                      float *dst32, int dst32_stride, int R, int H);
+cudaError_t reduce_splits(Launch L, SplitIn P, float *Y, int ldy, int R, int ncols);
+
+// gemm_simt.cu : Y[R][sum n_out] (fp32, ld ldy) = X[R][K_in] * W^T, X and W of `dtype`
+cudaError_t gemm_simt(Launch L, int dtype, const void *X, GemmMats m, int K_in, int R, float *Y,
+                      int ldy);
+
+// gemm_tc.cu : bf16 tensor-core path; writes `split` partial matrices `split_stride` apart.
+int tc_init_driver(char *err, size_t errlen);   // 0 on success
+bool tc_supported(const GemmMats &m, int K_in);
+int tc_default_split(int n_tiles, int kblocks);
+cudaError_t gemm_tc(Launch L, const void *X, int x_rows_alloc, GemmMats m, int K_in, int R,
+                    float *Y, int ldy, int split, size_t split_stride, int *status);
+
+// tree.cu
+struct TreeBufs {
+  int32_t *tree_tok, *tree_parent, *tree_level, *tree_n;
+  float *tree_score;
+  uint64_t *tree_anc;      // [B][N][2]
+  int32_t *cand_tok, *cand_parent, *cand_level, *cand_rank;
+  float *cand_score;
+  int32_t *frontier;       // [B][k] candidate ids
+  uint64_t *front_mask;    // [B][k][2] draft-cache visibility of each frontier row
+  int32_t *front_row;      // [B][pool] draft tree row of a candidate once it was a frontier row
+  int32_t *topk_tok;
+  float *topk_logp;
+  int32_t *root_tok, *pend_tok, *n_pend, *acc_path, *acc_len, *acc_S;
+  float *pend_hid;
+};
+struct PlanBufs {
+  int32_t *pos, *slot, *ctx_len, *kv_len, *row_src, *row_tok, *last_row;
+  uint64_t *mask;
+  float2 *rope;
+};
+cudaError_t tree_from_caller(Launch L, TreeBufs t, const int32_t *tok, const int32_t *parent,
+                             const int32_t *n_nodes, int stride, int B, int N, int *status);
+cudaError_t tree_ancestors(Launch L, TreeBufs t, int B, int N);
+cudaError_t plan_verify(Launch L, TreeBufs t, PlanBufs p, const int32_t *seq_len, int B, int N,
+                        int head_dim, float rope_base, int S_max, int *status);
+cudaError_t plan_draft0(Launch L, TreeBufs t, PlanBufs p, const int32_t *seq_len, int B, int N,
+                        int rows, int head_dim, float rope_base, int S_max, int *status);
+cudaError_t plan_draft_p(Launch L, TreeBufs t, PlanBufs p, const int32_t *seq_len, int B, int k,
+                         int pool, int pass, int head_dim, float rope_base, int S_max, int *status);
+cudaError_t expand_dynamic(Launch L, TreeBufs t, int B, int k, int pool, int pass, int D, int N);
+cudaError_t expand_static(Launch L, TreeBufs t, const int32_t *s_parent, const int32_t *s_level,
+                          const int32_t *s_rank, int B, int N, int k);
+cudaError_t plan_medusa(Launch L, TreeBufs t, PlanBufs p, int B, int N, int heads);
+cudaError_t accept_walk(Launch L, TreeBufs t, const int32_t *verify_tgt, const float *verify_hid,
+                        const int32_t *forced_len, int32_t *seq_len, int32_t *out_tokens,
+                        int out_stride, int32_t *out_len, int B, int N, int H);
+cudaError_t kv_compact(Launch L, int dtype, TreeBufs t, void *k_cache, void *v_cache, int L_layers,
+                       int B, int N, int n_heads, int head_dim, int S_max);
+
+}  // namespace koala

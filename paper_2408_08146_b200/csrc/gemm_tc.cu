@@ -1,0 +1,412 @@
+// Weight-streaming skinny GEMM on the 5th-generation tensor cores (sm_100a):
+//   Y[R][N_out] (fp32) = X[R][K_in] (bf16) * W[N_out][K_in]^T (bf16)
+// with R (tokens = tree nodes x batch) small and the weight matrix read exactly once.
+//
+// Operands are swapped so that the weights fill the MMA's M dimension: one CTA owns 128 weight
+// rows and a range of K, and issues tcgen05.mma with M = 128 (weight rows), N = token tile,
+// K = 16, both operands K-major in shared memory with the 128-byte swizzle that TMA writes.
+// The fp32 accumulator [128 x tokens] lives in tensor memory.  Warp 0 streams weight and
+// activation tiles with TMA through a ring of shared-memory stages (mbarrier full/empty pairs),
+// warp 1 issues the MMAs, warps 2..5 read the accumulator back (tcgen05.ld) and store it.
+// The weight stream does not depend on the previous kernel, so under programmatic dependent
+// launch the first stages are requested before waiting for the producer of X.
+// Split-K: grid.y CTAs share a weight tile and write separate partial outputs that the consumer
+// kernel sums in a fixed order (deterministic).
+// Every wait is bounded: on expiry the kernel records KOALA_E_TIMEOUT in *status, drains, frees
+// its tensor memory and returns.
+#include <cuda.h>
+
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <tuple>
+
+#include "common.cuh"
+
+namespace koala {
+namespace {
+
+constexpr int BM = 128;             // weight rows per CTA (MMA M)
+constexpr int BK = 64;              // K elements per stage: 128 bytes of bf16 = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int THREADS = 192;
+constexpr int W_STAGE_BYTES = BM * BK * 2;
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // about a second of SM clock
+constexpr int E_TIMEOUT = 6;
+constexpr int MAX_STAGES = 12;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+               "r"(bytes)
+               : "memory");
+}
+// Bounded wait; returns false if the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+  const uint32_t addr = smem_u32(bar);
+  const long long t0 = clock64();
+  while (true) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) return false;
+  }
+}
+__device__ __forceinline__ void tma_load_2d(const CUtensorMap *map, uint64_t *bar, void *dst, int x,
+                                            int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 bytes apart,
+// 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address
+  d |= (uint64_t)1 << 16;                          // leading byte offset (unused for this layout)
+  d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                          // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                          // 128-byte swizzle
+  return d;
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t *v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+        "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+        "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+struct TcParams {
+  float *Y;
+  int ldy;
+  int R;              // valid tokens
+  int bn;             // token tile (MMA N), multiple of 16, <= 256
+  int tmem_cols;      // power of two >= max(32, bn)
+  int tiles0, tiles1; // weight tiles of matrix 0 and of matrices 0+1 (cumulative)
+  int n0, n1, n2;     // rows of each matrix
+  int kblocks;        // K_in / 64
+  int split;          // CTAs along K
+  size_t split_stride;
+  int stages;
+  int *status;
+};
+
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
+               const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX,
+               const TcParams P) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ uint64_t full_bar[MAX_STAGES];
+  __shared__ uint64_t empty_bar[MAX_STAGES];
+  __shared__ uint64_t accum_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int s_error;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t raw = smem_u32(smem_raw);
+  unsigned char *tiles = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+  const int x_stage_bytes = P.bn * BK * 2;
+  const int stage_bytes = W_STAGE_BYTES + x_stage_bytes;   // both multiples of 1024 (bn % 16 == 0 -> x multiple of 2048)
+
+  // which matrix / which rows
+  int tile = blockIdx.x;
+  const CUtensorMap *tmW = &tmW0;
+  int col_off = 0, n_rows = P.n0;
+  if (tile >= P.tiles1) { tmW = &tmW2; tile -= P.tiles1; col_off = P.n0 + P.n1; n_rows = P.n2; }
+  else if (tile >= P.tiles0) { tmW = &tmW1; tile -= P.tiles0; col_off = P.n0; n_rows = P.n1; }
+  const int row0 = tile * BM;
+  const int tok0 = blockIdx.z * P.bn;
+  // K range of this split
+  const int kb_lo = (int)(((long long)P.kblocks * blockIdx.y) / P.split);
+  const int kb_hi = (int)(((long long)P.kblocks * (blockIdx.y + 1)) / P.split);
+  const int nkb = kb_hi - kb_lo;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < P.stages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(&accum_bar, 1);
+    s_error = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)P.tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_acc = tmem_base_slot;
+  pdl_launch_dependents();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(tmW) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
+      const int pre = nkb < P.stages ? nkb : P.stages;
+      // weights first: they do not depend on the kernel before this one
+      for (int it = 0; it < pre; ++it) {
+        mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
+        tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, (kb_lo + it) * BK, row0);
+      }
+      pdl_wait();
+      for (int it = 0; it < pre; ++it)
+        tma_load_2d(&tmX, &full_bar[it], tiles + (size_t)it * stage_bytes + W_STAGE_BYTES,
+                    (kb_lo + it) * BK, tok0);
+      bool ok = true;
+      for (int it = pre; it < nkb && ok; ++it) {
+        const int s = it % P.stages;
+        const uint32_t ph = (uint32_t)(it / P.stages) & 1u;
+        ok = mbar_wait(&empty_bar[s], ph ^ 1u);
+        if (!ok) break;
+        mbar_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
+        unsigned char *dst = tiles + (size_t)s * stage_bytes;
+        tma_load_2d(tmW, &full_bar[s], dst, (kb_lo + it) * BK, row0);
+        tma_load_2d(&tmX, &full_bar[s], dst + W_STAGE_BYTES, (kb_lo + it) * BK, tok0);
+      }
+      if (!ok) {
+        atomicExch(&s_error, 1);
+        // let the copies already requested land before the block's memory goes away
+        for (int s = 0; s < P.stages; ++s) (void)mbar_wait(&full_bar[s], 0);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: D fp32, A and B bf16, both K-major, N = bn, M = 128
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.bn >> 3) << 17) |
+                             ((uint32_t)(BM >> 4) << 24);
+      bool ok = true;
+      for (int it = 0; it < nkb; ++it) {
+        const int s = it % P.stages;
+        const uint32_t ph = (uint32_t)(it / P.stages) & 1u;
+        ok = mbar_wait(&full_bar[s], ph);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t wa = smem_u32(tiles + (size_t)s * stage_bytes);
+        const uint64_t da = smem_desc_sw128(wa);
+        const uint64_t db = smem_desc_sw128(wa + W_STAGE_BYTES);
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; ++k) {
+          // advance 32 bytes (16 bf16) inside the swizzled row: +2 in the 16-byte address field
+          umma_bf16(tmem_acc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
+                    (it > 0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
+      }
+      if (ok) umma_commit(&accum_bar);   // accumulator complete
+      else atomicExch(&s_error, 1);
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;        // the 32 tensor-memory lanes this warp may read
+    pdl_wait();                          // the output buffer may still be read by the previous kernel
+    bool ok = true;
+    if (nkb > 0) ok = mbar_wait(&accum_bar, 0);
+    if (!ok) atomicExch(&s_error, 1);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int feat = row0 + quarter * 32 + lane;
+    float *Yp = P.Y + (size_t)blockIdx.y * P.split_stride + col_off + feat;
+    if (ok) {
+      for (int c0 = 0; c0 < P.bn; c0 += 16) {
+        uint32_t v[16];
+        if (nkb > 0) {
+          tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = 0u;
+        }
+        if (feat < n_rows) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int t = tok0 + c0 + j;
+            if (t < P.R) Yp[(size_t)t * P.ldy] = __uint_as_float(v[j]);
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                 ::"r"(tmem_acc), "r"((uint32_t)P.tmem_cols)
+                 : "memory");
+  }
+  if (threadIdx.x == 0 && s_error && P.status) atomicMax(P.status, E_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+std::mutex g_mu;
+std::map<std::tuple<const void *, int, int, int>, CUtensorMap> g_maps;   // (ptr, rows, K, box rows)
+int g_smem_optin = 0;
+int g_num_sms = 148;
+
+bool get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  auto key = std::make_tuple(ptr, rows, K_in, box_rows);
+  auto it = g_maps.find(key);
+  if (it != g_maps.end()) {
+    *out = it->second;
+    return true;
+  }
+  if (!g_encode) return false;
+  CUtensorMap m;
+  cuuint64_t dims[2] = {(cuuint64_t)K_in, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K_in * 2};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides,
+                        box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  g_maps[key] = m;
+  *out = m;
+  return true;
+}
+
+}  // namespace
+
+int tc_init_driver(char *err, size_t errlen) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  if (g_encode) return 0;
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+  if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || fn == nullptr) {
+    snprintf(err, errlen, "cuTensorMapEncodeTiled not available: %s", cudaGetErrorString(e));
+    return 1;
+  }
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&g_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+  e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g_smem_optin - 1024);
+  if (e != cudaSuccess) {
+    snprintf(err, errlen, "cannot raise the GEMM kernel's shared memory: %s", cudaGetErrorString(e));
+    return 1;
+  }
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return 0;
+}
+
+void tc_forget_maps() {
+  std::lock_guard<std::mutex> lock(g_mu);
+  g_maps.clear();
+}
+
+bool tc_supported(const GemmMats &m, int K_in) {
+  if (K_in % BK != 0 || K_in < BK) return false;
+  for (int i = 0; i < m.n; ++i)
+    if (m.n_out[i] < 1 || ((uintptr_t)m.W[i] & 15u)) return false;
+  return g_encode != nullptr;
+}
+
+// Split so that tiles x split comes close to a whole number of waves of the SMs, while every
+// split keeps at least 8 K-blocks.
+int tc_default_split(int n_tiles, int kblocks) {
+  int best = 1;
+  double best_eff = 0.0;
+  const int max_split = kblocks / 8 > 0 ? (kblocks / 8 < 16 ? kblocks / 8 : 16) : 1;
+  for (int s = 1; s <= max_split; ++s) {
+    const int ctas = n_tiles * s;
+    const int waves = (ctas + g_num_sms - 1) / g_num_sms;
+    const double eff = (double)ctas / ((double)waves * g_num_sms);
+    if (eff > best_eff + 0.03) {
+      best_eff = eff;
+      best = s;
+    }
+  }
+  return best;
+}
+
+cudaError_t gemm_tc(Launch L, const void *X, int x_rows_alloc, GemmMats m, int K_in, int R,
+                    float *Y, int ldy, int split, size_t split_stride, int *status) {
+  if (!tc_supported(m, K_in) || R < 1) return cudaErrorInvalidValue;
+  TcParams P;
+  memset(&P, 0, sizeof(P));
+  int bn = ((R + 15) / 16) * 16;
+  if (bn > 256) bn = 256;
+  if (bn > x_rows_alloc) return cudaErrorInvalidValue;
+  int cols = 32;
+  while (cols < bn) cols <<= 1;
+  P.Y = Y;
+  P.ldy = ldy;
+  P.R = R;
+  P.bn = bn;
+  P.tmem_cols = cols;
+  const int t0 = (m.n_out[0] + BM - 1) / BM;
+  const int t1 = m.n > 1 ? (m.n_out[1] + BM - 1) / BM : 0;
+  const int t2 = m.n > 2 ? (m.n_out[2] + BM - 1) / BM : 0;
+  P.tiles0 = t0;
+  P.tiles1 = t0 + t1;
+  P.n0 = m.n_out[0];
+  P.n1 = m.n > 1 ? m.n_out[1] : 0;
+  P.n2 = m.n > 2 ? m.n_out[2] : 0;
+  P.kblocks = K_in / BK;
+  if (split < 1) split = 1;
+  if (split > P.kblocks) split = P.kblocks;
+  P.split = split;
+  P.split_stride = split_stride;
+  P.status = status;
+  const int stage_bytes = W_STAGE_BYTES + bn * BK * 2;
+  int stages = (g_smem_optin - 2048) / stage_bytes;
+  if (stages > MAX_STAGES) stages = MAX_STAGES;
+  if (stages > 8) stages = 8;
+  if (stages < 2) return cudaErrorInvalidValue;
+  P.stages = stages;
+  CUtensorMap mw[3], mx;
+  for (int i = 0; i < 3; ++i) {
+    const int j = i < m.n ? i : 0;
+    if (!get_map(m.W[j], m.n_out[j], K_in, BM, &mw[i])) return cudaErrorInvalidValue;
+  }
+  if (!get_map(X, x_rows_alloc, K_in, bn, &mx)) return cudaErrorInvalidValue;
+  dim3 grid(t0 + t1 + t2, split, (R + bn - 1) / bn);
+  const size_t smem = (size_t)stages * stage_bytes + 1024;
+  return launch_k(gemm_tc_kernel, grid, dim3(THREADS), smem, L.st, L.pdl, mw[0], mw[1], mw[2], mx, P);
+}
+
+}  // namespace koala

@@ -1,0 +1,613 @@
+// C ABI of libkoala: context, workspace carving and the kernel sequence of each step.
+// Host code only enqueues kernels on the caller's stream; it never synchronises.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/koala.h"
+#include "common.cuh"
+
+using namespace koala;
+
+namespace koala {
+void tc_forget_maps();
+}
+
+namespace {
+
+enum Phase { PH_READY = 0, PH_DRAFTED, PH_EXPANDED, PH_TREE, PH_VERIFIED };
+
+struct LayerW {
+  const void *attn_norm, *wq, *wk, *wv, *wo, *ffn_norm, *wg, *wu, *wd;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Walks the workspace; with base == nullptr it only measures.
+struct Carver {
+  unsigned char *base;
+  size_t off;
+  template <typename T> T *take(size_t count) {
+    off = align_up(off, 256);
+    T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+constexpr int MAX_SPLIT = 8;
+
+}  // namespace
+
+struct koala_ctx {
+  koala_config cfg;
+  cudaStream_t st;
+  bool pdl, use_tc;
+  const void *embed, *lm_head, *final_norm, *fc_w, *fc_b;
+  std::vector<LayerW> layers, draft_layers;
+  std::vector<const void *> res_w, res_b;
+  void *tk, *tv, *dk, *dv;
+  int32_t *seq_len;
+  // derived sizes
+  int M, Mp, pool, draft_rows_max, esz;
+  size_t pcols;           // widest GEMM output
+  // workspace
+  float *x, *qbuf, *P, *verify_logits, *draft_logits, *verify_hid, *feat[2], *mx;
+  void *xn, *attn_out, *act, *cat, *lmin;
+  int32_t *verify_tgt, *s_parent, *s_level, *s_rank;
+  int *status;
+  TreeBufs t;
+  PlanBufs p;
+  // host state
+  Phase phase;
+  int last_pass, pend_cap, draft_rows;
+  bool last_tree_from_caller;
+  int *host_status;       // pinned
+  cudaEvent_t poll_ev;
+  bool poll_pending;
+  int last_status;
+  char err[256];
+};
+
+namespace {
+
+int fail(koala_ctx *c, int code, const char *fmt, ...) {
+  if (c) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(c->err, sizeof(c->err), fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+#define CU_TRY(expr)                                                                     \
+  do {                                                                                   \
+    cudaError_t e__ = (expr);                                                            \
+    if (e__ != cudaSuccess)                                                              \
+      return fail(c, KOALA_E_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__));     \
+  } while (0)
+
+bool config_ok(const koala_config *cfg, char *why, size_t n) {
+#define BAD(msg)              \
+  do {                        \
+    snprintf(why, n, msg);    \
+    return false;             \
+  } while (0)
+  if (!cfg) BAD("null config");
+  if (cfg->struct_size != sizeof(koala_config)) BAD("koala_config.struct_size mismatch");
+  if (cfg->dtype != KOALA_FP32 && cfg->dtype != KOALA_BF16) BAD("dtype must be fp32 or bf16");
+  if (cfg->head_kind != KOALA_EAGLE && cfg->head_kind != KOALA_MEDUSA) BAD("unknown head_kind");
+  if (cfg->L < 1 || cfg->H < 1 || cfg->F < 1 || cfg->V < 2) BAD("non-positive model dimension");
+  if (cfg->n_heads < 1 || cfg->n_heads * cfg->head_dim != cfg->H) BAD("n_heads * head_dim != H");
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) BAD("head_dim must be 64 or 128");
+  if (cfg->K < 0 || cfg->K > 64) BAD("K out of range");
+  if (cfg->topk < 1 || cfg->topk > KOALA_MAX_TOPK || cfg->topk > cfg->V) BAD("topk out of range");
+  if (cfg->N < 1 || cfg->N > KOALA_MAX_TREE) BAD("N out of range");
+  if (cfg->B < 1 || cfg->B > 64) BAD("B out of range");
+  if (cfg->D < 1 || cfg->D > 16) BAD("D out of range");
+  if (cfg->S_max < cfg->N) BAD("S_max smaller than the tree");
+  if (cfg->head_kind == KOALA_MEDUSA) {
+    if (cfg->n_medusa_heads < 1 || cfg->n_medusa_heads > 16) BAD("n_medusa_heads out of range");
+    if (cfg->D != cfg->n_medusa_heads) BAD("MEDUSA: D must equal n_medusa_heads");
+  } else {
+    if ((cfg->D - 1) * cfg->topk > 128) BAD("EAGLE: (D-1)*topk must be <= 128");
+  }
+  if (!(cfg->rms_eps > 0.f) || !(cfg->rope_base > 1.f)) BAD("bad rms_eps / rope_base");
+#undef BAD
+  return true;
+}
+
+// Assigns (or measures) every workspace buffer.  Must visit the same sequence in both modes.
+size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
+  Carver w{base, 0};
+  const int B = cfg.B, N = cfg.N, H = cfg.H, F = cfg.F, V = cfg.V, k = cfg.topk;
+  const int M = B * N;
+  int draft_rows = B * k;
+  if (cfg.head_kind == KOALA_MEDUSA && cfg.n_medusa_heads * B > draft_rows) draft_rows = cfg.n_medusa_heads * B;
+  int rows = M > draft_rows ? M : draft_rows;
+  const int Mp = (int)align_up((size_t)rows + 16, 16);
+  const int pool = cfg.head_kind == KOALA_EAGLE ? k + (cfg.D - 1) * k * k : k;
+  const size_t pcols = (size_t)(3 * H > 2 * F ? 3 * H : 2 * F);
+  const size_t esz = cfg.dtype == KOALA_FP32 ? 4 : 2;
+  c->M = M; c->Mp = Mp; c->pool = pool; c->draft_rows_max = draft_rows; c->esz = (int)esz; c->pcols = pcols;
+  c->x = w.take<float>((size_t)Mp * H);
+  c->qbuf = w.take<float>((size_t)Mp * H);
+  c->P = w.take<float>((size_t)MAX_SPLIT * Mp * pcols);
+  c->verify_logits = w.take<float>((size_t)Mp * V);
+  c->draft_logits = w.take<float>((size_t)(draft_rows + 16) * V);
+  c->verify_hid = w.take<float>((size_t)Mp * H);
+  c->feat[0] = w.take<float>((size_t)(B * k + 16) * H);
+  c->feat[1] = w.take<float>((size_t)(B * k + 16) * H);
+  c->mx = w.take<float>((size_t)Mp * H);
+  c->xn = w.take<unsigned char>((size_t)Mp * H * esz);
+  c->attn_out = w.take<unsigned char>((size_t)Mp * H * esz);
+  c->act = w.take<unsigned char>((size_t)Mp * F * esz);
+  c->cat = w.take<unsigned char>((size_t)Mp * 2 * H * esz);
+  c->lmin = w.take<unsigned char>((size_t)Mp * H * esz);
+  c->verify_tgt = w.take<int32_t>(Mp);
+  c->s_parent = w.take<int32_t>(N);
+  c->s_level = w.take<int32_t>(N);
+  c->s_rank = w.take<int32_t>(N);
+  c->status = w.take<int>(4);
+  TreeBufs &t = c->t;
+  t.tree_tok = w.take<int32_t>(M);
+  t.tree_parent = w.take<int32_t>(M);
+  t.tree_level = w.take<int32_t>(M);
+  t.tree_n = w.take<int32_t>(B);
+  t.tree_score = w.take<float>(M);
+  t.tree_anc = w.take<uint64_t>((size_t)M * 2);
+  t.cand_tok = w.take<int32_t>((size_t)B * pool);
+  t.cand_parent = w.take<int32_t>((size_t)B * pool);
+  t.cand_level = w.take<int32_t>((size_t)B * pool);
+  t.cand_rank = w.take<int32_t>((size_t)B * pool);
+  t.cand_score = w.take<float>((size_t)B * pool);
+  t.frontier = w.take<int32_t>((size_t)B * k);
+  t.front_mask = w.take<uint64_t>((size_t)B * k * 2);
+  t.front_row = w.take<int32_t>((size_t)B * pool);
+  t.topk_tok = w.take<int32_t>((size_t)draft_rows * k);
+  t.topk_logp = w.take<float>((size_t)draft_rows * k);
+  t.root_tok = w.take<int32_t>(B);
+  t.pend_tok = w.take<int32_t>(M);
+  t.n_pend = w.take<int32_t>(B);
+  t.acc_path = w.take<int32_t>(M);
+  t.acc_len = w.take<int32_t>(B);
+  t.acc_S = w.take<int32_t>(B);
+  t.pend_hid = w.take<float>((size_t)M * H);
+  PlanBufs &p = c->p;
+  p.pos = w.take<int32_t>(Mp);
+  p.slot = w.take<int32_t>(Mp);
+  p.ctx_len = w.take<int32_t>(B);
+  p.kv_len = w.take<int32_t>(B);
+  p.row_src = w.take<int32_t>(Mp);
+  p.row_tok = w.take<int32_t>(Mp);
+  p.last_row = w.take<int32_t>(B);
+  p.mask = w.take<uint64_t>((size_t)Mp * 2);
+  p.rope = w.take<float2>((size_t)Mp * (cfg.head_dim / 2));
+  return align_up(w.off, 256);
+}
+
+Launch LN(koala_ctx *c) { return Launch{c->st, c->pdl}; }
+
+RowPlan row_plan(koala_ctx *c) {
+  return RowPlan{c->p.pos, c->p.slot, c->p.mask, c->p.ctx_len, c->p.kv_len, c->p.rope};
+}
+
+// Y = X * [W...]^T as a (possibly split) fp32 result in the partial buffer, or directly into
+// `direct` (ld = ld_direct) when given.
+int do_gemm(koala_ctx *c, const void *X, int K_in, GemmMats m, int R, float *direct, int ld_direct,
+            SplitIn *out) {
+  int ncols = 0;
+  for (int i = 0; i < m.n; ++i) ncols += m.n_out[i];
+  float *Y = direct ? direct : c->P;
+  const int ld = direct ? ld_direct : ncols;
+  if (c->use_tc && c->cfg.dtype == KOALA_BF16 && tc_supported(m, K_in)) {
+    int tiles = 0;
+    for (int i = 0; i < m.n; ++i) tiles += (m.n_out[i] + 127) / 128;
+    int split = direct ? 1 : tc_default_split(tiles, K_in / 64);
+    if (split > MAX_SPLIT) split = MAX_SPLIT;
+    const size_t stride = (size_t)c->Mp * ld;
+    CU_TRY(gemm_tc(LN(c), X, c->Mp, m, K_in, R, Y, ld, split, stride, c->status));
+    if (out) *out = SplitIn{Y, split, stride, ld};
+  } else {
+    CU_TRY(gemm_simt(LN(c), c->cfg.dtype, X, m, K_in, R, Y, ld));
+    if (out) *out = SplitIn{Y, 1, 0, ld};
+  }
+  return KOALA_OK;
+}
+
+#define K_TRY(expr)              \
+  do {                           \
+    int rc__ = (expr);           \
+    if (rc__ != KOALA_OK) return rc__; \
+  } while (0)
+
+// One pre-norm decoder layer over R rows.  On entry x holds the residual stream and xn the
+// normalised input of the attention block.  On exit x is updated and `next_xn` holds
+// T(rmsnorm(x) * next_g) (or T(x) if next_g is null); `out_f32` optionally receives the same in fp32.
+int run_layer(koala_ctx *c, const LayerW &w, void *kc, void *vc, int R, int rows_per_seq,
+              const void *next_g, void *next_xn, float *out_f32) {
+  const koala_config &g = c->cfg;
+  const int H = g.H, F = g.F;
+  SplitIn s;
+  GemmMats qkv{{w.wq, w.wk, w.wv}, {H, H, H}, 3};
+  K_TRY(do_gemm(c, c->xn, H, qkv, R, nullptr, 0, &s));
+  CU_TRY(rope_kv_write(LN(c), g.dtype, s, row_plan(c), c->qbuf, kc, vc, R, rows_per_seq, g.n_heads,
+                       g.head_dim, g.S_max));
+  CU_TRY(tree_attention(LN(c), g.dtype, c->qbuf, kc, vc, row_plan(c), c->attn_out, R, rows_per_seq, g.B,
+                        g.n_heads, g.head_dim, g.S_max));
+  GemmMats o{{w.wo, nullptr, nullptr}, {H, 0, 0}, 1};
+  K_TRY(do_gemm(c, c->attn_out, H, o, R, nullptr, 0, &s));
+  CU_TRY(row_epilogue(LN(c), g.dtype, 0, c->x, s, nullptr, w.ffn_norm, c->xn, nullptr, R, H, g.rms_eps));
+  GemmMats gu{{w.wg, w.wu, nullptr}, {F, F, 0}, 2};
+  K_TRY(do_gemm(c, c->xn, H, gu, R, nullptr, 0, &s));
+  CU_TRY(swiglu(LN(c), g.dtype, s, c->act, R, F));
+  GemmMats dn{{w.wd, nullptr, nullptr}, {H, 0, 0}, 1};
+  K_TRY(do_gemm(c, c->act, F, dn, R, nullptr, 0, &s));
+  CU_TRY(row_epilogue(LN(c), g.dtype, 0, c->x, s, nullptr, next_g, next_xn, out_f32, R, H, g.rms_eps));
+  return KOALA_OK;
+}
+
+size_t kv_layer_elems(const koala_config &g) {
+  return (size_t)g.B * g.n_heads * g.S_max * g.head_dim;
+}
+
+int draft_eagle(koala_ctx *c, int pass) {
+  const koala_config &g = c->cfg;
+  const int H = g.H, k = g.topk, B = g.B;
+  const int rows = pass == 0 ? c->pend_cap : k;
+  const int R = B * rows;
+  const float *feat_src;
+  if (pass == 0) {
+    CU_TRY(plan_draft0(LN(c), c->t, c->p, c->seq_len, B, g.N, rows, g.head_dim, g.rope_base, g.S_max,
+                       c->status));
+    feat_src = c->t.pend_hid;
+  } else {
+    CU_TRY(plan_draft_p(LN(c), c->t, c->p, c->seq_len, B, k, c->pool, pass, g.head_dim, g.rope_base,
+                        g.S_max, c->status));
+    feat_src = c->feat[(pass - 1) & 1];
+  }
+  CU_TRY(eagle_concat(LN(c), g.dtype, feat_src, c->p.row_src, c->p.row_tok, c->embed, c->cat, R, H, g.V));
+  SplitIn s;
+  GemmMats fc{{c->fc_w, nullptr, nullptr}, {H, 0, 0}, 1};
+  K_TRY(do_gemm(c, c->cat, 2 * H, fc, R, nullptr, 0, &s));
+  // pass 0: the feature of every row stays in x and the last valid row is gathered afterwards;
+  // pass >= 1: every row's feature goes to feat[pass & 1] and to the LM head's input.
+  float *f_all = pass == 0 ? nullptr : c->feat[pass & 1];
+  void *lm_all = pass == 0 ? nullptr : c->lmin;
+  if (g.K == 0) {
+    CU_TRY(row_epilogue(LN(c), g.dtype, 1, c->x, s, c->fc_b, nullptr, lm_all, f_all, R, H, g.rms_eps));
+  } else {
+    CU_TRY(row_epilogue(LN(c), g.dtype, 1, c->x, s, c->fc_b, c->draft_layers[0].attn_norm, c->xn, nullptr,
+                        R, H, g.rms_eps));
+    const size_t le = kv_layer_elems(g) * c->esz;
+    for (int j = 0; j < g.K; ++j) {
+      const bool last = j == g.K - 1;
+      K_TRY(run_layer(c, c->draft_layers[j], (unsigned char *)c->dk + j * le, (unsigned char *)c->dv + j * le,
+                      R, rows, last ? nullptr : c->draft_layers[j + 1].attn_norm, last ? lm_all : c->xn,
+                      last ? f_all : nullptr));
+    }
+  }
+  int lm_rows = R;
+  if (pass == 0) {
+    CU_TRY(cast_rows(LN(c), g.dtype, c->x, c->p.last_row, c->lmin, c->feat[0], k, B, H));
+    lm_rows = B;
+  }
+  GemmMats lm{{c->lm_head, nullptr, nullptr}, {g.V, 0, 0}, 1};
+  K_TRY(do_gemm(c, c->lmin, H, lm, lm_rows, c->draft_logits, g.V, nullptr));
+  c->draft_rows = lm_rows;
+  return KOALA_OK;
+}
+
+int draft_medusa(koala_ctx *c) {
+  const koala_config &g = c->cfg;
+  const int H = g.H, B = g.B, nh = g.n_medusa_heads;
+  const int R = nh * B;
+  CU_TRY(plan_medusa(LN(c), c->t, c->p, B, g.N, nh));
+  CU_TRY(cast_rows(LN(c), g.dtype, c->t.pend_hid, c->p.row_src, c->xn, c->mx, 1, R, H));
+  for (int j = 0; j < g.K; ++j) {
+    for (int i = 0; i < nh; ++i) {
+      SplitIn s;
+      GemmMats m{{c->res_w[(size_t)i * g.K + j], nullptr, nullptr}, {H, 0, 0}, 1};
+      unsigned char *xi = (unsigned char *)c->xn + (size_t)i * B * H * c->esz;
+      K_TRY(do_gemm(c, xi, H, m, B, nullptr, 0, &s));
+      CU_TRY(row_epilogue(LN(c), g.dtype, 2, c->mx + (size_t)i * B * H, s, c->res_b[(size_t)i * g.K + j],
+                          nullptr, xi, nullptr, B, H, g.rms_eps));
+    }
+  }
+  GemmMats lm{{c->lm_head, nullptr, nullptr}, {g.V, 0, 0}, 1};
+  K_TRY(do_gemm(c, c->xn, H, lm, R, c->draft_logits, g.V, nullptr));
+  c->draft_rows = R;
+  return KOALA_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+extern "C" {
+#pragma GCC visibility push(default)
+
+size_t koala_workspace_bytes(const koala_config *cfg) {
+  char why[128];
+  if (!config_ok(cfg, why, sizeof(why))) return 0;
+  koala_ctx tmp;
+  return carve(&tmp, *cfg, nullptr);
+}
+
+int koala_init(const koala_config *cfg, const koala_weights *w, const koala_state *st,
+               void *cuda_stream, koala_ctx **out) {
+  if (!out) return KOALA_E_INVALID;
+  *out = nullptr;
+  koala_ctx *c = new (std::nothrow) koala_ctx();
+  if (!c) return KOALA_E_INVALID;
+  *out = c;   // returned even on failure so that koala_last_error() can be read; destroy it either way
+  c->err[0] = 0;
+  c->host_status = nullptr;
+  c->poll_ev = nullptr;
+  c->poll_pending = false;
+  c->last_status = 0;
+  char why[128];
+  if (!config_ok(cfg, why, sizeof(why))) return fail(c, KOALA_E_INVALID, "%s", why);
+  if (!w || !st) return fail(c, KOALA_E_INVALID, "null weights or state");
+  c->cfg = *cfg;
+  const koala_config &g = c->cfg;
+  if (!w->embed || !w->lm_head || !w->final_norm || !w->layer_w)
+    return fail(c, KOALA_E_INVALID, "missing target weights");
+  if (!st->target_k || !st->target_v || !st->seq_len || !st->workspace)
+    return fail(c, KOALA_E_INVALID, "missing state pointers");
+  if (((uintptr_t)st->workspace & 255u) != 0) return fail(c, KOALA_E_INVALID, "workspace not 256-byte aligned");
+  c->st = (cudaStream_t)cuda_stream;
+  c->pdl = (g.flags & KOALA_F_NO_PDL) == 0;
+  c->use_tc = (g.flags & KOALA_F_NO_TENSOR_CORES) == 0 && g.dtype == KOALA_BF16;
+  c->embed = w->embed;
+  c->lm_head = w->lm_head;
+  c->final_norm = w->final_norm;
+  c->fc_w = w->fc_w;
+  c->fc_b = w->fc_b;
+  auto fill_layers = [](std::vector<LayerW> &dst, const void *const *src, int n) {
+    dst.resize(n);
+    for (int l = 0; l < n; ++l) {
+      const void *const *q = src + (size_t)l * KOALA_LAYER_TENSORS;
+      dst[l] = LayerW{q[0], q[1], q[2], q[3], q[4], q[5], q[6], q[7], q[8]};
+      for (int i = 0; i < KOALA_LAYER_TENSORS; ++i)
+        if (!q[i]) return false;
+    }
+    return true;
+  };
+  if (!fill_layers(c->layers, w->layer_w, g.L)) return fail(c, KOALA_E_INVALID, "null target layer tensor");
+  if (g.head_kind == KOALA_EAGLE) {
+    if (!w->fc_w || !w->fc_b || (g.K > 0 && (!w->draft_layer_w || !st->draft_k || !st->draft_v)))
+      return fail(c, KOALA_E_INVALID, "missing EAGLE head weights or cache");
+    if (g.K > 0 && !fill_layers(c->draft_layers, w->draft_layer_w, g.K))
+      return fail(c, KOALA_E_INVALID, "null draft layer tensor");
+  } else {
+    if (!w->static_parent || !w->static_level || !w->static_rank)
+      return fail(c, KOALA_E_INVALID, "missing static tree");
+    if (g.K > 0 && (!w->res_w || !w->res_b)) return fail(c, KOALA_E_INVALID, "missing Medusa blocks");
+    const int n = g.n_medusa_heads * g.K;
+    c->res_w.assign(w->res_w, w->res_w + n);
+    c->res_b.assign(w->res_b, w->res_b + n);
+    for (int i = 0; i < n; ++i)
+      if (!c->res_w[i] || !c->res_b[i]) return fail(c, KOALA_E_INVALID, "null Medusa block tensor");
+    for (int u = 0; u < g.N; ++u) {
+      const int p = w->static_parent[u], lv = w->static_level[u], rk = w->static_rank[u];
+      const bool ok = u == 0 ? (p == -1 && lv == 0)
+                             : (p >= 0 && p < u && lv == w->static_level[p] + 1 && lv <= g.n_medusa_heads &&
+                                rk >= 0 && rk < g.topk);
+      if (!ok) return fail(c, KOALA_E_INVALID, "malformed static tree at node %d", u);
+    }
+  }
+  c->tk = st->target_k; c->tv = st->target_v; c->dk = st->draft_k; c->dv = st->draft_v;
+  c->seq_len = st->seq_len;
+  const size_t need = carve(c, g, (unsigned char *)st->workspace);
+  if (st->workspace_bytes < need)
+    return fail(c, KOALA_E_CAPACITY, "workspace too small: %zu < %zu bytes", st->workspace_bytes, need);
+  if (c->use_tc) {
+    char e[160];
+    if (tc_init_driver(e, sizeof(e)) != 0) return fail(c, KOALA_E_CUDA, "%s", e);
+  }
+  // small state that must start at zero
+  CU_TRY(cudaMemsetAsync(c->status, 0, 4 * sizeof(int), c->st));
+  CU_TRY(cudaMemsetAsync(c->t.n_pend, 0, g.B * sizeof(int32_t), c->st));
+  CU_TRY(cudaMemsetAsync(c->t.root_tok, 0, g.B * sizeof(int32_t), c->st));
+  CU_TRY(cudaMemsetAsync(c->t.tree_n, 0, g.B * sizeof(int32_t), c->st));
+  if (g.head_kind == KOALA_MEDUSA) {
+    CU_TRY(cudaMemcpyAsync(c->s_parent, w->static_parent, g.N * sizeof(int32_t), cudaMemcpyHostToDevice, c->st));
+    CU_TRY(cudaMemcpyAsync(c->s_level, w->static_level, g.N * sizeof(int32_t), cudaMemcpyHostToDevice, c->st));
+    CU_TRY(cudaMemcpyAsync(c->s_rank, w->static_rank, g.N * sizeof(int32_t), cudaMemcpyHostToDevice, c->st));
+    // the copies above read pageable host arrays: they are staged before the call returns
+  }
+  CU_TRY(cudaHostAlloc((void **)&c->host_status, sizeof(int), cudaHostAllocDefault));
+  *c->host_status = 0;
+  CU_TRY(cudaEventCreateWithFlags(&c->poll_ev, cudaEventDisableTiming));
+  c->phase = PH_READY;
+  c->last_pass = -1;
+  c->pend_cap = g.N < g.D + 1 ? g.N : g.D + 1;
+  c->draft_rows = 0;
+  c->last_tree_from_caller = false;
+  return KOALA_OK;
+}
+
+int koala_draft(koala_ctx *c, int pass) {
+  if (!c) return KOALA_E_INVALID;
+  const koala_config &g = c->cfg;
+  if (g.head_kind == KOALA_MEDUSA) {
+    if (pass != 0) return fail(c, KOALA_E_INVALID, "Medusa-style heads draft in the single pass 0");
+    if (c->phase != PH_READY) return fail(c, KOALA_E_STATE, "koala_draft(0) must follow koala_init / koala_accept");
+    K_TRY(draft_medusa(c));
+  } else {
+    if (pass < 0 || pass >= g.D) return fail(c, KOALA_E_INVALID, "pass %d outside 0..D-1", pass);
+    if (pass == 0 && c->phase != PH_READY)
+      return fail(c, KOALA_E_STATE, "koala_draft(0) must follow koala_init / koala_accept");
+    if (pass > 0 && !(c->phase == PH_EXPANDED && c->last_pass == pass - 1))
+      return fail(c, KOALA_E_STATE, "koala_draft(%d) must follow koala_expand_tree(%d)", pass, pass - 1);
+    K_TRY(draft_eagle(c, pass));
+  }
+  c->phase = PH_DRAFTED;
+  c->last_pass = pass;
+  return KOALA_OK;
+}
+
+int koala_expand_tree(koala_ctx *c, int pass) {
+  if (!c) return KOALA_E_INVALID;
+  const koala_config &g = c->cfg;
+  if (c->phase != PH_DRAFTED || c->last_pass != pass)
+    return fail(c, KOALA_E_STATE, "koala_expand_tree(%d) must follow koala_draft(%d)", pass, pass);
+  CU_TRY(topk_logp(LN(c), c->draft_logits, c->t.topk_tok, c->t.topk_logp, c->draft_rows, g.V, g.topk));
+  if (g.head_kind == KOALA_MEDUSA) {
+    CU_TRY(expand_static(LN(c), c->t, c->s_parent, c->s_level, c->s_rank, g.B, g.N, g.topk));
+    c->phase = PH_TREE;
+  } else {
+    CU_TRY(expand_dynamic(LN(c), c->t, g.B, g.topk, c->pool, pass, g.D, g.N));
+    c->phase = pass == g.D - 1 ? PH_TREE : PH_EXPANDED;
+  }
+  return KOALA_OK;
+}
+
+int koala_verify(koala_ctx *c, const koala_tree *tree) {
+  if (!c) return KOALA_E_INVALID;
+  const koala_config &g = c->cfg;
+  if (tree) {
+    if (!tree->tok || !tree->parent || !tree->n_nodes) return fail(c, KOALA_E_INVALID, "null tree arrays");
+    if (tree->n_max < 1 || tree->n_max > g.N || tree->stride < tree->n_max)
+      return fail(c, KOALA_E_INVALID, "tree n_max %d / stride %d out of range (N = %d)", tree->n_max,
+                  tree->stride, g.N);
+    CU_TRY(tree_from_caller(LN(c), c->t, tree->tok, tree->parent, tree->n_nodes, tree->stride, g.B, g.N,
+                            c->status));
+    c->last_tree_from_caller = true;
+    c->pend_cap = tree->n_max;
+  } else {
+    if (c->phase != PH_TREE) return fail(c, KOALA_E_STATE, "no drafted tree: run draft/expand_tree first");
+    c->last_tree_from_caller = false;
+    c->pend_cap = g.N < g.D + 1 ? g.N : g.D + 1;
+  }
+  const int R = g.B * g.N;
+  CU_TRY(tree_ancestors(LN(c), c->t, g.B, g.N));
+  CU_TRY(plan_verify(LN(c), c->t, c->p, c->seq_len, g.B, g.N, g.head_dim, g.rope_base, g.S_max, c->status));
+  CU_TRY(embed_norm(LN(c), g.dtype, c->p.row_tok, c->embed, c->layers[0].attn_norm, c->x, c->xn, R, g.H, g.V,
+                    g.rms_eps));
+  const size_t le = kv_layer_elems(g) * c->esz;
+  for (int l = 0; l < g.L; ++l) {
+    const bool last = l == g.L - 1;
+    K_TRY(run_layer(c, c->layers[l], (unsigned char *)c->tk + l * le, (unsigned char *)c->tv + l * le, R, g.N,
+                    last ? c->final_norm : c->layers[l + 1].attn_norm, last ? c->lmin : c->xn,
+                    last ? c->verify_hid : nullptr));
+  }
+  GemmMats lm{{c->lm_head, nullptr, nullptr}, {g.V, 0, 0}, 1};
+  K_TRY(do_gemm(c, c->lmin, g.H, lm, R, c->verify_logits, g.V, nullptr));
+  CU_TRY(argmax_rows(LN(c), c->verify_logits, c->verify_tgt, R, g.V));
+  c->phase = PH_VERIFIED;
+  return KOALA_OK;
+}
+
+int koala_accept(koala_ctx *c, const int32_t *forced_len, int32_t *out_tokens, int32_t out_stride,
+                 int32_t *out_len) {
+  if (!c) return KOALA_E_INVALID;
+  const koala_config &g = c->cfg;
+  if (!out_tokens || !out_len || out_stride < 1) return fail(c, KOALA_E_INVALID, "null outputs");
+  if (c->phase != PH_VERIFIED) return fail(c, KOALA_E_STATE, "koala_accept must follow koala_verify");
+  CU_TRY(accept_walk(LN(c), c->t, c->verify_tgt, c->verify_hid, forced_len, c->seq_len, out_tokens,
+                     out_stride, out_len, g.B, g.N, g.H));
+  CU_TRY(kv_compact(LN(c), g.dtype, c->t, c->tk, c->tv, g.L, g.B, g.N, g.n_heads, g.head_dim, g.S_max));
+  c->phase = PH_READY;
+  c->last_pass = -1;
+  return KOALA_OK;
+}
+
+int koala_buffers(koala_ctx *c, koala_buffer_table *o) {
+  if (!c || !o) return KOALA_E_INVALID;
+  memset(o, 0, sizeof(*o));
+  o->draft_logits = c->draft_logits;
+  o->draft_feat = c->cfg.head_kind == KOALA_MEDUSA ? c->mx : c->feat[c->last_pass >= 0 ? (c->last_pass & 1) : 0];
+  o->topk_tok = c->t.topk_tok;
+  o->topk_logp = c->t.topk_logp;
+  o->cand_tok = c->t.cand_tok;
+  o->cand_parent = c->t.cand_parent;
+  o->cand_score = c->t.cand_score;
+  o->frontier = c->t.frontier;
+  o->tree_tok = c->t.tree_tok;
+  o->tree_parent = c->t.tree_parent;
+  o->tree_level = c->t.tree_level;
+  o->tree_score = c->t.tree_score;
+  o->tree_n = c->t.tree_n;
+  o->verify_logits = c->verify_logits;
+  o->verify_hid = c->verify_hid;
+  o->verify_tgt = c->verify_tgt;
+  o->root_tok = c->t.root_tok;
+  o->pend_hid = c->t.pend_hid;
+  o->pend_tok = c->t.pend_tok;
+  o->n_pend = c->t.n_pend;
+  o->acc_path = c->t.acc_path;
+  o->pool = c->pool;
+  o->draft_rows = c->draft_rows;
+  return KOALA_OK;
+}
+
+int koala_poll(koala_ctx *c, int *done, int *device_status) {
+  if (!c) return KOALA_E_INVALID;
+  if (c->poll_pending && cudaEventQuery(c->poll_ev) == cudaSuccess) {
+    c->last_status = *c->host_status;
+    c->poll_pending = false;
+  }
+  if (!c->poll_pending) {
+    CU_TRY(cudaMemcpyAsync(c->host_status, c->status, sizeof(int), cudaMemcpyDeviceToHost, c->st));
+    CU_TRY(cudaEventRecord(c->poll_ev, c->st));
+    c->poll_pending = true;
+    if (cudaEventQuery(c->poll_ev) == cudaSuccess) {
+      c->last_status = *c->host_status;
+      c->poll_pending = false;
+    }
+  }
+  if (done) *done = c->poll_pending ? 0 : 1;
+  if (device_status) *device_status = c->last_status;
+  (void)cudaGetLastError();
+  return KOALA_OK;
+}
+
+const char *koala_last_error(const koala_ctx *c) { return c ? c->err : "null context"; }
+
+void koala_destroy(koala_ctx *c) {
+  if (!c) return;
+  if (c->host_status) cudaFreeHost(c->host_status);
+  if (c->poll_ev) cudaEventDestroy(c->poll_ev);
+  koala::tc_forget_maps();
+  delete c;
+}
+
+size_t koala_gemm_scratch_bytes(int M, int N_out, int K_in) {
+  (void)K_in;
+  if (M < 1 || N_out < 1) return 0;
+  return (size_t)MAX_SPLIT * ((size_t)M + 16) * (size_t)N_out * sizeof(float);
+}
+
+int koala_gemm_bf16(const void *X, const void *W, float *Y, int ldy, int M, int N_out, int K_in,
+                    void *scratch, size_t scratch_bytes, int use_tensor_cores, int split_k,
+                    void *cuda_stream, int *device_status) {
+  if (!X || !W || !Y || M < 1 || N_out < 1 || K_in < 1 || ldy < N_out) return KOALA_E_INVALID;
+  Launch L{(cudaStream_t)cuda_stream, false};
+  GemmMats m{{W, nullptr, nullptr}, {N_out, 0, 0}, 1};
+  if (!use_tensor_cores) return gemm_simt(L, KOALA_BF16, X, m, K_in, M, Y, ldy) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
+  char e[160];
+  if (tc_init_driver(e, sizeof(e)) != 0) return KOALA_E_CUDA;
+  if (!tc_supported(m, K_in)) return KOALA_E_UNSUPPORTED;
+  int split = split_k > 0 ? split_k : tc_default_split((N_out + 127) / 128, K_in / 64);
+  if (split > MAX_SPLIT) split = MAX_SPLIT;
+  if (split > K_in / 64) split = K_in / 64;
+  // X must hold a whole token tile: the caller's buffer has M rows, rounded up by the map's
+  // out-of-bounds zero fill
+  const int rows_alloc = ((M + 15) / 16) * 16;
+  if (split == 1) {
+    return gemm_tc(L, X, rows_alloc, m, K_in, M, Y, ldy, 1, 0, device_status) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
+  }
+  const size_t stride = (size_t)M * N_out;
+  if (!scratch || scratch_bytes < (size_t)split * stride * sizeof(float)) return KOALA_E_CAPACITY;
+  if (gemm_tc(L, X, rows_alloc, m, K_in, M, (float *)scratch, N_out, split, stride, device_status) != cudaSuccess)
+    return KOALA_E_CUDA;
+  SplitIn s{(const float *)scratch, split, stride, N_out};
+  return reduce_splits(L, s, Y, ldy, M, N_out) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

@@ -1,0 +1,403 @@
+// Row-wise kernels of the decoder layers and heads: embedding gather, RMSNorm / residual
+// epilogues, RoPE + KV-cache write, SwiGLU, tree-masked attention (CUDA-core version),
+// arg-max and top-k with log-probabilities.  All statistics are fp32.
+#include "common.cuh"
+
+namespace koala {
+
+namespace {
+
+__device__ __forceinline__ float block_sum(float v, float *red) {
+  v = warp_sum(v);
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  if (lane == 0) red[w] = v;
+  __syncthreads();
+  float t = (threadIdx.x < nw) ? red[threadIdx.x] : 0.f;
+  if (w == 0) {
+    t = warp_sum(t);
+    if (lane == 0) red[0] = t;
+  }
+  __syncthreads();
+  t = red[0];
+  __syncthreads();
+  return t;
+}
+
+__device__ __forceinline__ float silu_f(float v) { return v / (1.f + expf(-v)); }
+
+// ------------------------------------------------------------------------------- embedding + norm
+template <typename T>
+__global__ void embed_norm_kernel(const int32_t *__restrict__ tok, const T *__restrict__ E,
+                                  const T *__restrict__ g, float *__restrict__ x,
+                                  T *__restrict__ xn, int H, int V, float eps) {
+  __shared__ float red[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  int t = tok[r];
+  t = t < 0 ? 0 : (t >= V ? V - 1 : t);
+  const T *e = E + (size_t)t * H;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < H; i += blockDim.x) {
+    const float v = to_f(e[i]);
+    x[(size_t)r * H + i] = v;
+    ss += v * v;
+  }
+  const float inv = rsqrtf(block_sum(ss, red) / (float)H + eps);
+  for (int i = threadIdx.x; i < H; i += blockDim.x)
+    xn[(size_t)r * H + i] = from_f<T>(x[(size_t)r * H + i] * inv * to_f(g[i]));
+}
+
+// ------------------------------------------------------------------------------- row epilogue
+template <typename T>
+__global__ void row_epilogue_kernel(int mode, float *__restrict__ x, SplitIn P,
+                                    const T *__restrict__ bias, const T *__restrict__ g,
+                                    T *__restrict__ xn, float *__restrict__ out_f32, int H,
+                                    float eps) {
+  __shared__ float red[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  float *xr = x + (size_t)r * H;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < H; i += blockDim.x) {
+    float p = P.at(r, i);
+    float v;
+    if (mode == 0) v = xr[i] + p;
+    else if (mode == 1) v = p + to_f(bias[i]);
+    else v = xr[i] + silu_f(p + to_f(bias[i]));
+    xr[i] = v;
+    ss += v * v;
+  }
+  float inv = 1.f;
+  if (g != nullptr) inv = rsqrtf(block_sum(ss, red) / (float)H + eps);
+  for (int i = threadIdx.x; i < H; i += blockDim.x) {
+    float n = xr[i];
+    if (g != nullptr) n = n * inv * to_f(g[i]);
+    if (xn != nullptr) xn[(size_t)r * H + i] = from_f<T>(n);
+    if (out_f32 != nullptr) out_f32[(size_t)r * H + i] = n;
+  }
+}
+
+// ------------------------------------------------------------------------------- EAGLE fc input
+template <typename T>
+__global__ void eagle_concat_kernel(const float *__restrict__ feat_src,
+                                    const int32_t *__restrict__ row_src,
+                                    const int32_t *__restrict__ row_tok, const T *__restrict__ E,
+                                    T *__restrict__ cat, int H, int V) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  const int src = row_src[r];
+  int t = row_tok[r];
+  t = t < 0 ? 0 : (t >= V ? V - 1 : t);
+  const float *f = feat_src + (size_t)src * H;
+  const T *e = E + (size_t)t * H;
+  T *c = cat + (size_t)r * 2 * H;
+  for (int i = threadIdx.x; i < H; i += blockDim.x) {
+    c[i] = from_f<T>(f[i]);
+    c[H + i] = e[i];
+  }
+}
+
+template <typename T>
+__global__ void cast_rows_kernel(const float *__restrict__ src, const int32_t *__restrict__ row_src,
+                                 T *__restrict__ dst, float *__restrict__ dst32, int dst32_stride,
+                                 int H) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  const int s = row_src ? row_src[r] : r;
+  for (int i = threadIdx.x; i < H; i += blockDim.x) {
+    const float v = src[(size_t)s * H + i];
+    dst[(size_t)r * H + i] = from_f<T>(v);
+    if (dst32) dst32[(size_t)r * dst32_stride * H + i] = v;
+  }
+}
+
+__global__ void reduce_splits_kernel(SplitIn P, float *__restrict__ Y, int ldy, int ncols) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.y;
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c < ncols) Y[(size_t)r * ldy + c] = P.at(r, c);
+}
+
+// ------------------------------------------------------------------------------- RoPE + KV write
+// grid (R, n_heads), block head_dim/2: thread i rotates the pair (i, i + head_dim/2).
+template <typename T>
+__global__ void rope_kv_kernel(SplitIn qkv, RowPlan plan, float *__restrict__ q_out,
+                               T *__restrict__ k_cache, T *__restrict__ v_cache, int rows_per_seq,
+                               int n_heads, int head_dim, int S_max) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x, h = blockIdx.y, i = threadIdx.x;
+  const int half = head_dim >> 1, H = n_heads * head_dim;
+  const int b = r / rows_per_seq;
+  const int slot = plan.slot[r];
+  const float2 cs = plan.rope[(size_t)r * half + i];
+  const int c0 = h * head_dim + i, c1 = c0 + half;
+  const float q0 = qkv.at(r, c0), q1 = qkv.at(r, c1);
+  q_out[(size_t)r * H + c0] = q0 * cs.x - q1 * cs.y;
+  q_out[(size_t)r * H + c1] = q1 * cs.x + q0 * cs.y;
+  if (slot < 0 || slot >= S_max) return;
+  const float k0 = qkv.at(r, H + c0), k1 = qkv.at(r, H + c1);
+  const float v0 = qkv.at(r, 2 * H + c0), v1 = qkv.at(r, 2 * H + c1);
+  const size_t base = (((size_t)b * n_heads + h) * S_max + slot) * head_dim;
+  k_cache[base + i] = from_f<T>(k0 * cs.x - k1 * cs.y);
+  k_cache[base + i + half] = from_f<T>(k1 * cs.x + k0 * cs.y);
+  v_cache[base + i] = from_f<T>(v0);
+  v_cache[base + i + half] = from_f<T>(v1);
+}
+
+// ------------------------------------------------------------------------------- SwiGLU
+template <typename T>
+__global__ void swiglu_kernel(SplitIn gu, T *__restrict__ act, int F) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.y;
+  const int f = blockIdx.x * blockDim.x + threadIdx.x;
+  if (f >= F) return;
+  act[(size_t)r * F + f] = from_f<T>(silu_f(gu.at(r, f)) * gu.at(r, F + f));
+}
+
+// ------------------------------------------------------------------------------- tree attention
+// One block = 8 query rows of one (sequence, head); one warp per query row.  Keys/values stream
+// through shared memory 32 at a time; lane j scores key j, then the warp accumulates P.V with
+// each lane owning DH/32 output dimensions.  Online softmax in fp32.
+template <typename T, int DH>
+__global__ void __launch_bounds__(256)
+tree_attn_kernel(const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc,
+                 RowPlan plan, T *__restrict__ out, int rows_per_seq, int n_heads, int S_max) {
+  __shared__ float Ks[32][DH + 1];
+  __shared__ float Vs[32][DH];
+  __shared__ float qs[8][DH];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int b = blockIdx.z, h = blockIdx.y;
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int i = blockIdx.x * 8 + w;
+  const int H = n_heads * DH;
+  const int r = b * rows_per_seq + (i < rows_per_seq ? i : 0);
+  const bool valid = (i < rows_per_seq) && (plan.slot[r] >= 0);
+  const int ctx = plan.ctx_len[b], kv_len = plan.kv_len[b];
+  const uint64_t m0 = plan.mask[(size_t)r * 2], m1 = plan.mask[(size_t)r * 2 + 1];
+  for (int d = lane; d < DH; d += 32) qs[w][d] = valid ? q[(size_t)r * H + h * DH + d] : 0.f;
+  const T *kb = kc + ((size_t)b * n_heads + h) * S_max * DH;
+  const T *vb = vc + ((size_t)b * n_heads + h) * S_max * DH;
+  const float scale = rsqrtf((float)DH);
+  float m = -INFINITY, l = 0.f;
+  float o[DH / 32];
+#pragma unroll
+  for (int d = 0; d < DH / 32; ++d) o[d] = 0.f;
+  for (int t0 = 0; t0 < kv_len; t0 += 32) {
+    __syncthreads();
+    for (int e = threadIdx.x; e < 32 * DH; e += 256) {
+      const int j = e / DH, d = e % DH;
+      const bool in = (t0 + j) < kv_len;
+      Ks[j][d] = in ? to_f(kb[(size_t)(t0 + j) * DH + d]) : 0.f;
+      Vs[j][d] = in ? to_f(vb[(size_t)(t0 + j) * DH + d]) : 0.f;
+    }
+    __syncthreads();
+    const int t = t0 + lane;
+    bool vis = valid && t < kv_len;
+    if (vis && t >= ctx) {
+      const int rel = t - ctx;
+      vis = rel < 64 ? ((m0 >> rel) & 1ull) : (rel < 128 ? ((m1 >> (rel - 64)) & 1ull) : false);
+    }
+    float s = 0.f;
+#pragma unroll 8
+    for (int d = 0; d < DH; ++d) s += qs[w][d] * Ks[lane][d];
+    s = vis ? s * scale : -INFINITY;
+    const float m_new = fmaxf(m, warp_max(s));
+    if (m_new == -INFINITY) continue;   // nothing visible so far (uniform across the warp)
+    const float p = vis ? expf(s - m_new) : 0.f;
+    const float corr = (m == -INFINITY) ? 0.f : expf(m - m_new);
+    l = l * corr + warp_sum(p);
+    m = m_new;
+#pragma unroll
+    for (int d = 0; d < DH / 32; ++d) o[d] *= corr;
+    for (int j = 0; j < 32; ++j) {
+      const float pj = __shfl_sync(0xffffffffu, p, j);
+#pragma unroll
+      for (int d = 0; d < DH / 32; ++d) o[d] += pj * Vs[j][lane + 32 * d];
+    }
+  }
+  if (i < rows_per_seq) {
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+    for (int d = 0; d < DH / 32; ++d)
+      out[(size_t)r * H + h * DH + lane + 32 * d] = from_f<T>(o[d] * inv);
+  }
+}
+
+// ------------------------------------------------------------------------------- arg-max / top-k
+struct ValIdx {
+  float v;
+  int i;
+};
+__device__ __forceinline__ ValIdx better(ValIdx a, ValIdx b) {
+  return (b.v > a.v || (b.v == a.v && b.i < a.i)) ? b : a;
+}
+__device__ __forceinline__ ValIdx block_argmax(ValIdx x, ValIdx *red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    ValIdx y;
+    y.v = __shfl_xor_sync(0xffffffffu, x.v, o);
+    y.i = __shfl_xor_sync(0xffffffffu, x.i, o);
+    x = better(x, y);
+  }
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  if (lane == 0) red[w] = x;
+  __syncthreads();
+  if (w == 0) {
+    ValIdx y = lane < nw ? red[lane] : ValIdx{-INFINITY, 0x7fffffff};
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      ValIdx z;
+      z.v = __shfl_xor_sync(0xffffffffu, y.v, o);
+      z.i = __shfl_xor_sync(0xffffffffu, y.i, o);
+      y = better(y, z);
+    }
+    if (lane == 0) red[0] = y;
+  }
+  __syncthreads();
+  x = red[0];
+  __syncthreads();
+  return x;
+}
+
+__global__ void argmax_rows_kernel(const float *__restrict__ logits, int32_t *__restrict__ out, int V) {
+  __shared__ ValIdx red[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const float *row = logits + (size_t)blockIdx.x * V;
+  ValIdx best{-INFINITY, 0x7fffffff};
+  for (int i = threadIdx.x; i < V; i += blockDim.x) best = better(best, ValIdx{row[i], i});
+  best = block_argmax(best, red);
+  if (threadIdx.x == 0) out[blockIdx.x] = best.i;
+}
+
+// Per row: the k largest logits (ties: smaller id) and their natural-log softmax probabilities.
+// The row is staged in shared memory; each round removes the current maximum.
+__global__ void topk_logp_kernel(const float *__restrict__ logits, int32_t *__restrict__ tok,
+                                 float *__restrict__ logp, int V, int k) {
+  extern __shared__ float srow[];
+  __shared__ ValIdx red[32];
+  __shared__ float redf[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const float *row = logits + (size_t)blockIdx.x * V;
+  ValIdx best{-INFINITY, 0x7fffffff};
+  for (int i = threadIdx.x; i < V; i += blockDim.x) {
+    const float v = row[i];
+    srow[i] = v;
+    best = better(best, ValIdx{v, i});
+  }
+  best = block_argmax(best, red);
+  const float mx = best.v;
+  float se = 0.f;
+  for (int i = threadIdx.x; i < V; i += blockDim.x) se += expf(srow[i] - mx);
+  const float lse = mx + logf(block_sum(se, redf));
+  for (int j = 0; j < k; ++j) {
+    if (j > 0) {
+      best = ValIdx{-INFINITY, 0x7fffffff};
+      for (int i = threadIdx.x; i < V; i += blockDim.x) best = better(best, ValIdx{srow[i], i});
+      best = block_argmax(best, red);
+    }
+    if (threadIdx.x == 0) {
+      tok[(size_t)blockIdx.x * k + j] = best.i;
+      logp[(size_t)blockIdx.x * k + j] = best.v - lse;
+      srow[best.i] = -INFINITY;
+    }
+    __syncthreads();
+  }
+}
+
+}  // namespace
+
+#define DISPATCH_T(dtype, ...)                \
+  if ((dtype) == 0) {                         \
+    typedef float T;                          \
+    __VA_ARGS__                               \
+  } else {                                    \
+    typedef bf16 T;                           \
+    __VA_ARGS__                               \
+  }
+
+cudaError_t embed_norm(Launch L, int dtype, const int32_t *tok, const void *E, const void *g,
+                       float *x, void *xn, int R, int H, int V, float eps) {
+  DISPATCH_T(dtype, return launch_k(embed_norm_kernel<T>, dim3(R), dim3(256), 0, L.st, L.pdl, tok,
+                                    (const T *)E, (const T *)g, x, (T *)xn, H, V, eps);)
+}
+
+cudaError_t row_epilogue(Launch L, int dtype, int mode, float *x, SplitIn P, const void *bias,
+                         const void *g, void *xn, float *out_f32, int R, int H, float eps) {
+  DISPATCH_T(dtype, return launch_k(row_epilogue_kernel<T>, dim3(R), dim3(256), 0, L.st, L.pdl, mode,
+                                    x, P, (const T *)bias, (const T *)g, (T *)xn, out_f32, H, eps);)
+}
+
+cudaError_t eagle_concat(Launch L, int dtype, const float *feat_src, const int32_t *row_src,
+                         const int32_t *row_tok, const void *E, void *cat, int R, int H, int V) {
+  DISPATCH_T(dtype, return launch_k(eagle_concat_kernel<T>, dim3(R), dim3(256), 0, L.st, L.pdl,
+                                    feat_src, row_src, row_tok, (const T *)E, (T *)cat, H, V);)
+}
+
+cudaError_t cast_rows(Launch L, int dtype, const float *src, const int32_t *row_src, void *dst,
+                      float *dst32, int dst32_stride, int R, int H) {
+  DISPATCH_T(dtype, return launch_k(cast_rows_kernel<T>, dim3(R), dim3(256), 0, L.st, L.pdl, src,
+                                    row_src, (T *)dst, dst32, dst32_stride, H);)
+}
+
+cudaError_t reduce_splits(Launch L, SplitIn P, float *Y, int ldy, int R, int ncols) {
+  return launch_k(reduce_splits_kernel, dim3((ncols + 255) / 256, R), dim3(256), 0, L.st, L.pdl, P, Y,
+                  ldy, ncols);
+}
+
+cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowPlan plan, float *q_out,
+                          void *k_cache, void *v_cache, int R, int rows_per_seq, int n_heads,
+                          int head_dim, int S_max) {
+  DISPATCH_T(dtype, return launch_k(rope_kv_kernel<T>, dim3(R, n_heads), dim3(head_dim / 2), 0, L.st,
+                                    L.pdl, qkv, plan, q_out, (T *)k_cache, (T *)v_cache,
+                                    rows_per_seq, n_heads, head_dim, S_max);)
+}
+
+cudaError_t swiglu(Launch L, int dtype, SplitIn gu, void *act, int R, int F) {
+  DISPATCH_T(dtype, return launch_k(swiglu_kernel<T>, dim3((F + 255) / 256, R), dim3(256), 0, L.st,
+                                    L.pdl, gu, (T *)act, F);)
+}
+
+cudaError_t tree_attention(Launch L, int dtype, const float *q, const void *k_cache,
+                           const void *v_cache, RowPlan plan, void *out, int R, int rows_per_seq,
+                           int B, int n_heads, int head_dim, int S_max) {
+  (void)R;
+  dim3 grid((rows_per_seq + 7) / 8, n_heads, B);
+  if (head_dim == 64) {
+    DISPATCH_T(dtype, return launch_k(tree_attn_kernel<T, 64>, grid, dim3(256), 0, L.st, L.pdl, q,
+                                      (const T *)k_cache, (const T *)v_cache, plan, (T *)out,
+                                      rows_per_seq, n_heads, S_max);)
+  } else if (head_dim == 128) {
+    DISPATCH_T(dtype, return launch_k(tree_attn_kernel<T, 128>, grid, dim3(256), 0, L.st, L.pdl, q,
+                                      (const T *)k_cache, (const T *)v_cache, plan, (T *)out,
+                                      rows_per_seq, n_heads, S_max);)
+  }
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t argmax_rows(Launch L, const float *logits, int32_t *out, int R, int V) {
+  return launch_k(argmax_rows_kernel, dim3(R), dim3(1024), 0, L.st, L.pdl, logits, out, V);
+}
+
+cudaError_t topk_logp(Launch L, const float *logits, int32_t *tok, float *logp, int R, int V, int k) {
+  const size_t smem = (size_t)V * sizeof(float);
+  static size_t configured = 0;
+  if (smem > 48 * 1024 && smem > configured) {
+    cudaError_t e = cudaFuncSetAttribute(topk_logp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = smem;
+  }
+  return launch_k(topk_logp_kernel, dim3(R), dim3(1024), smem, L.st, L.pdl, logits, tok, logp, V, k);
+}
+
+}  // namespace koala

@@ -1,0 +1,45 @@
+"""The library's matrix multiplies (tensor-core and CUDA-core paths) against a float64 product."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2408_08146_b200 import koala_gemm_bf16
+from workloads.generate import normal_tensor
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [  # (tokens, out features, in features)
+    (1, 128, 64), (10, 4096, 4096), (16, 256, 128), (17, 200, 192), (60, 1536, 4096),
+    (64, 384, 11008), (40, 640, 5120), (256, 256, 1024), (300, 256, 512), (6, 32000, 4096)]
+
+
+def _inputs(M, N, K):
+    x = normal_tensor(7, f"x{M}.{N}.{K}", (M, K), 1.0, 0.0, torch.bfloat16, "cuda:0")
+    w = normal_tensor(8, f"w{M}.{N}.{K}", (N, K), 0.02, 0.0, torch.bfloat16, "cuda:0")
+    ref = x.double().cpu().numpy() @ w.double().cpu().numpy().T
+    return x, w, ref
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("split", [0, 1, 3])
+def test_tensor_core_gemm(shape, split):
+    M, N, K = shape
+    if split > K // 64:
+        pytest.skip("fewer K blocks than splits")
+    x, w, ref = _inputs(M, N, K)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    y = koala_gemm_bf16(x, w, True, split, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, "a bounded device-side wait ran out"
+    err = np.abs(y.cpu().numpy() - ref).max()
+    assert err <= 2e-5 * np.sqrt(K) + 1e-6, f"max err {err}"      # fp32 accumulation of K products
+
+
+@pytest.mark.parametrize("shape", SHAPES[:8])
+def test_cuda_core_gemm(shape):
+    M, N, K = shape
+    x, w, ref = _inputs(M, N, K)
+    y = koala_gemm_bf16(x, w, False)
+    torch.cuda.synchronize()
+    err = np.abs(y.cpu().numpy() - ref).max()
+    assert err <= 2e-5 * np.sqrt(K) + 1e-6, f"max err {err}"
