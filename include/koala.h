@@ -22,7 +22,9 @@
  *     status word that koala_poll() copies back.
  *   - Matrices are row-major [out][in].  "dtype" is the storage type of weights, KV caches and
  *     matrix-multiply operands (fp32 or bf16); accumulation, softmax, norms and the residual
- *     stream are fp32 in both cases.
+ *     stream are fp32 in both cases.  With bf16 the activations entering a matrix multiply are
+ *     kept as two bf16 values (the rounded value and its rounding residual) unless
+ *     KOALA_F_BF16_ACTIVATIONS is set, so only the weights and the KV cache are rounded to bf16.
  *   - KV caches are laid out [layer][B][n_heads][S_max][head_dim].
  *   - A tree has at most N nodes per sequence, node 0 the root, parent index < child index.
  *     Node u of sequence b is row b*N + u of every per-node buffer.
@@ -54,6 +56,10 @@ extern "C" {
 /* flags */
 #define KOALA_F_NO_TENSOR_CORES 1u /* run every GEMM on the CUDA-core path (debugging / A-B checks) */
 #define KOALA_F_NO_PDL 2u          /* launch kernels without programmatic dependent launch         */
+#define KOALA_F_BF16_ACTIVATIONS 4u /* bf16 only: round matrix-multiply inputs to plain bf16 instead of
+                                       keeping them as a bf16 pair (value + rounding residual); halves
+                                       the tensor-core work, costs about 1e-2 relative accuracy over a
+                                       32-layer forward */
 
 #define KOALA_MAX_TREE 128 /* largest N: ancestor sets are 128-bit masks */
 #define KOALA_MAX_TOPK 16
@@ -183,6 +189,30 @@ int koala_accept(koala_ctx *ctx, const int32_t *forced_len, int32_t *out_tokens,
 
 int koala_buffers(koala_ctx *ctx, koala_buffer_table *out);
 
+/* Run-time options.  KOALA_OPT_EXPAND_MODE splits koala_expand_tree for step-by-step checks:
+ * 0 = top-k then tree bookkeeping (default); 1 = top-k only (the call may be repeated);
+ * 2 = tree bookkeeping only, from whatever topk_tok / topk_logp hold (e.g. values the caller wrote). */
+#define KOALA_OPT_EXPAND_MODE 1
+/* KOALA_OPT_TIMING: 1 = bracket every matrix-multiply and attention launch with CUDA events on the
+ * context's stream (this removes the launch overlap between neighbouring kernels, so it is for
+ * per-kernel measurement, not for timing whole steps) and reset the totals; 0 = off (default). */
+#define KOALA_OPT_TIMING 2
+int koala_set_option(koala_ctx *ctx, int option, int value);
+
+/* Totals since KOALA_OPT_TIMING was switched on, per kernel class.  Synchronises the stream. */
+#define KOALA_CLS_GEMM_TC 0   /* tensor-core (tcgen05) matrix multiplies */
+#define KOALA_CLS_GEMM_SIMT 1 /* CUDA-core matrix multiplies */
+#define KOALA_CLS_ATTENTION 2 /* tree-masked attention */
+typedef struct {
+  float ms[3];           /* summed device time between the bracketing events */
+  uint64_t bytes[3];     /* algorithmic bytes: weight bytes of each multiply; K/V bytes of each attention */
+  int32_t launches[3];
+} koala_timing;
+int koala_timing_read(koala_ctx *ctx, koala_timing *out);
+
+/* Kernels launched by the library in this process so far (all contexts). */
+uint64_t koala_launch_count(void);
+
 /* Non-blocking: *done = 1 if everything enqueued so far has finished; *device_status = the
  * device status word as of the last finished poll copy (0 = fine, else a KOALA_E_* code). */
 int koala_poll(koala_ctx *ctx, int *done, int *device_status);
@@ -194,11 +224,13 @@ void koala_destroy(koala_ctx *ctx);
  * Y[M][N_out] (fp32, row stride ldy) = X[M][K_in] (bf16) * W[N_out][K_in]^T (bf16), on the
  * tensor-core path (use_tensor_cores != 0; needs K_in % 64 == 0) or the CUDA-core path.
  * `scratch` (device, >= koala_gemm_scratch_bytes) holds split-K partial sums.  On the tensor-core
- * path X must be allocated with its row count rounded up to a multiple of 16 (the extra rows are
- * read, their results discarded) and X, W must be 16-byte aligned.  split_k 0 = automatic.
- * Asynchronous on `cuda_stream`. */
+ * path X (and X_lo) must be allocated with koala_gemm_x_rows(M, X_lo != NULL) rows: whole token
+ * tiles (the extra rows are read, their results discarded); X, X_lo and W must be 16-byte aligned.
+ * split_k 0 = automatic.  Asynchronous on `cuda_stream`. */
+int koala_gemm_x_rows(int M, int has_lo);
 size_t koala_gemm_scratch_bytes(int M, int N_out, int K_in);
-int koala_gemm_bf16(const void *X, const void *W, float *Y, int ldy, int M, int N_out, int K_in,
+int koala_gemm_bf16(const void *X, const void *X_lo /* optional residual of X, same shape; NULL = none */,
+                    const void *W, float *Y, int ldy, int M, int N_out, int K_in,
                     void *scratch, size_t scratch_bytes, int use_tensor_cores, int split_k,
                     void *cuda_stream, int *device_status /* device int, may be NULL */);
 

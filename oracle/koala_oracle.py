@@ -91,6 +91,18 @@ def top_k(values: np.ndarray, k: int) -> np.ndarray:
     return order[:k].astype(np.int64)
 
 
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even of float32 values to bfloat16 (8 significant bits), returned as float32.
+
+    Storage rounding of a bf16 KV cache: the paper does not state a numeric precision (Section 4.1
+    gives none); the bf16 configurations store weights and caches in bf16, and a value is rounded
+    to the storage type when it is written.
+    """
+    b = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    bias = ((b >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
+    return ((b + bias) & np.uint32(0xFFFF0000)).view(np.float32)
+
+
 def argmax_first(values: np.ndarray) -> int:
     """Index of the maximum; the smallest index among equal maxima."""
     return int(np.argmax(values))
@@ -131,12 +143,14 @@ class KoalaOracle:
          head_kind, n_medusa_heads, rms_eps, rope_base.
     weight: callable name -> numpy array ([out][in] matrices; names as in the workload module).
     static_tree: (parent, level, rank) arrays for the Medusa-style static topology.
+    kv_round: optional storage rounding applied to keys and values as they enter a cache.
     """
 
     def __init__(self, cfg, weight: Callable[[str], np.ndarray], dtype=np.float64,
-                 static_tree=None):
+                 static_tree=None, kv_round: Optional[Callable[[np.ndarray], np.ndarray]] = None):
         self.cfg = cfg
         self.dt = dtype
+        self.kv_round = kv_round        # storage rounding of the caches (round_to_bf16 for bf16 caches)
         self._w = weight
         B, L, K = cfg.B, cfg.L, cfg.K
         shape = (cfg.S_max, cfg.n_heads, cfg.head_dim)
@@ -186,6 +200,9 @@ class KoalaOracle:
         v = (h @ self.W(prefix + "wv").T).reshape(n, c.n_heads, c.head_dim)
         q = rope(q, pos, c.rope_base)
         k = rope(k, pos, c.rope_base)
+        if self.kv_round is not None:           # the caches hold values in their storage type
+            k = self.kv_round(k).astype(self.dt)
+            v = self.kv_round(v).astype(self.dt)
         k_cache[slots] = k
         v_cache[slots] = v
         scale = 1.0 / np.sqrt(float(c.head_dim))

@@ -20,7 +20,7 @@ ERR_NAMES = {0: "KOALA_OK", 1: "KOALA_E_INVALID", 2: "KOALA_E_UNSUPPORTED", 3: "
              4: "KOALA_E_STATE", 5: "KOALA_E_CUDA", 6: "KOALA_E_TIMEOUT"}
 KOALA_FP32, KOALA_BF16 = 0, 1
 KOALA_EAGLE, KOALA_MEDUSA = 0, 1
-KOALA_F_NO_TENSOR_CORES, KOALA_F_NO_PDL = 1, 2
+KOALA_F_NO_TENSOR_CORES, KOALA_F_NO_PDL, KOALA_F_BF16_ACTIVATIONS = 1, 2, 4
 LAYER_TENSORS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")
 
 
@@ -65,6 +65,10 @@ class koala_buffer_table(C.Structure):
         ("pool", C.c_int32), ("draft_rows", C.c_int32)]
 
 
+class koala_timing(C.Structure):
+    _fields_ = [("ms", C.c_float * 3), ("bytes", C.c_uint64 * 3), ("launches", C.c_int32 * 3)]
+
+
 _lib = None
 
 
@@ -90,16 +94,24 @@ def load_library(rebuild: bool = False) -> C.CDLL:
     lib.koala_accept.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
     lib.koala_buffers.restype = C.c_int
     lib.koala_buffers.argtypes = [C.c_void_p, C.POINTER(koala_buffer_table)]
+    lib.koala_set_option.restype = C.c_int
+    lib.koala_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int]
+    lib.koala_timing_read.restype = C.c_int
+    lib.koala_timing_read.argtypes = [C.c_void_p, C.POINTER(koala_timing)]
+    lib.koala_launch_count.restype = C.c_uint64
+    lib.koala_launch_count.argtypes = []
     lib.koala_poll.restype = C.c_int
     lib.koala_poll.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     lib.koala_last_error.restype = C.c_char_p
     lib.koala_last_error.argtypes = [C.c_void_p]
     lib.koala_destroy.restype = None
     lib.koala_destroy.argtypes = [C.c_void_p]
+    lib.koala_gemm_x_rows.restype = C.c_int
+    lib.koala_gemm_x_rows.argtypes = [C.c_int, C.c_int]
     lib.koala_gemm_scratch_bytes.restype = C.c_size_t
     lib.koala_gemm_scratch_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
     lib.koala_gemm_bf16.restype = C.c_int
-    lib.koala_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
+    lib.koala_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_size_t, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
     _lib = lib
     return lib
@@ -132,25 +144,30 @@ def _i32_array(values) -> "C.Array":
 
 
 def koala_gemm_bf16(x: torch.Tensor, w: torch.Tensor, use_tensor_cores: bool = True, split_k: int = 0,
-                    status: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """Y[M][N] fp32 = x[M][K] (bf16) @ w[N][K]^T (bf16) through the library's GEMM."""
+                    status: Optional[torch.Tensor] = None, x_lo: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Y[M][N] fp32 = (x [+ x_lo])[M][K] (bf16) @ w[N][K]^T (bf16) through the library's GEMM."""
     lib = load_library()
     M, K = x.shape
     N = w.shape[0]
-    rows = (M + 15) // 16 * 16
+    rows = int(lib.koala_gemm_x_rows(M, int(x_lo is not None)))             # whole token tiles
     xp = torch.zeros(rows, K, dtype=torch.bfloat16, device=x.device)
     xp[:M] = x
+    xlp = None
+    if x_lo is not None:
+        xlp = torch.zeros(rows, K, dtype=torch.bfloat16, device=x.device)
+        xlp[:M] = x_lo
     y = torch.empty(M, N, dtype=torch.float32, device=x.device)
     nbytes = int(lib.koala_gemm_scratch_bytes(M, N, K))
     scratch = torch.empty(nbytes, dtype=torch.uint8, device=x.device)
     st = torch.cuda.current_stream(x.device).cuda_stream
-    rc = lib.koala_gemm_bf16(xp.data_ptr(), w.data_ptr(), y.data_ptr(), N, M, N, K, scratch.data_ptr(),
+    rc = lib.koala_gemm_bf16(xp.data_ptr(), xlp.data_ptr() if xlp is not None else None, w.data_ptr(),
+                             y.data_ptr(), N, M, N, K, scratch.data_ptr(),
                              nbytes, int(use_tensor_cores), split_k, st,
                              status.data_ptr() if status is not None else None)
     if rc != KOALA_OK:
         raise KoalaError(rc, "koala_gemm_bf16")
     # keep the operands alive until the stream has consumed them
-    y._koala_keep = (xp, scratch, w)
+    y._koala_keep = (xp, xlp, scratch, w)
     return y
 
 
@@ -245,6 +262,23 @@ class Koala:
                                           self.out_tokens.data_ptr(), self.out_stride, self.out_len.data_ptr()))
         self._keep_forced = forced_len
         return self.out_tokens, self.out_len
+
+    def set_expand_mode(self, mode: int):
+        self._check(self.lib.koala_set_option(self._ctx, 1, mode))
+
+    def set_timing(self, on: bool):
+        self._check(self.lib.koala_set_option(self._ctx, 2, int(on)))
+
+    def timing(self) -> Dict[str, Dict[str, float]]:
+        """Per kernel class: summed milliseconds, algorithmic bytes, launches (synchronises)."""
+        t = koala_timing()
+        self._check(self.lib.koala_timing_read(self._ctx, C.byref(t)))
+        names = ("gemm_tc", "gemm_simt", "attention")
+        return {n: {"ms": float(t.ms[i]), "bytes": int(t.bytes[i]), "launches": int(t.launches[i])}
+                for i, n in enumerate(names)}
+
+    def launch_count(self) -> int:
+        return int(self.lib.koala_launch_count())
 
     def poll(self):
         done, status = C.c_int(0), C.c_int(0)

@@ -59,6 +59,8 @@ struct RowPlan {
   const float2 *rope;     // [R][head_dim/2] (cos, sin)
 };
 
+extern unsigned long long g_launches;   // kernels launched by the library (defined in koala_api.cu)
+
 template <typename... KArgs, typename... Args>
 static inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
                                    cudaStream_t stream, bool pdl, Args... args) {
@@ -72,6 +74,7 @@ static inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block
   attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  ++g_launches;
   return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
@@ -83,6 +86,13 @@ struct Launch {
   bool pdl;
 };
 
+// A matrix-multiply operand in the storage dtype.  For bf16 `lo` holds the rounding residual of
+// `hi` (operand value = hi + lo); for fp32, or when the residual is not kept, lo is null.
+struct Operand {
+  void *hi;
+  void *lo;
+};
+
 struct GemmMats {         // up to three weight matrices sharing K_in, outputs concatenated
   const void *W[3];
   int n_out[3];
@@ -91,36 +101,36 @@ struct GemmMats {         // up to three weight matrices sharing K_in, outputs c
 
 // ops.cu
 cudaError_t embed_norm(Launch L, int dtype, const int32_t *tok, const void *E, const void *g,
-                       float *x, void *xn, int R, int H, int V, float eps);
+                       float *x, Operand xn, int R, int H, int V, float eps);
 // mode 0: v = x + sum(P); 1: v = sum(P) + bias; 2: v = x + SiLU(sum(P) + bias).  x <- v;
 // n = g ? rmsnorm(v) * g : v;  xn <- T(n) if xn;  out_f32 <- n if out_f32.
 cudaError_t row_epilogue(Launch L, int dtype, int mode, float *x, SplitIn P, const void *bias,
-                         const void *g, void *xn, float *out_f32, int R, int H, float eps);
+                         const void *g, Operand xn, float *out_f32, int R, int H, float eps);
 cudaError_t eagle_concat(Launch L, int dtype, const float *feat_src, const int32_t *row_src,
-                         const int32_t *row_tok, const void *E, void *cat, int R, int H, int V);
+                         const int32_t *row_tok, const void *E, Operand cat, int R, int H, int V);
 cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowPlan plan, float *q_out,
                           void *k_cache, void *v_cache, int R, int rows_per_seq, int n_heads,
                           int head_dim, int S_max);
-cudaError_t swiglu(Launch L, int dtype, SplitIn gu, void *act, int R, int F);
+cudaError_t swiglu(Launch L, int dtype, SplitIn gu, Operand act, int R, int F);
 cudaError_t tree_attention(Launch L, int dtype, const float *q, const void *k_cache,
-                           const void *v_cache, RowPlan plan, void *out, int R, int rows_per_seq,
+                           const void *v_cache, RowPlan plan, Operand out, int R, int rows_per_seq,
                            int B, int n_heads, int head_dim, int S_max);
 cudaError_t argmax_rows(Launch L, const float *logits, int32_t *out, int R, int V);
 cudaError_t topk_logp(Launch L, const float *logits, int32_t *tok, float *logp, int R, int V, int k);
 // dst[r] = T(src[row_src ? row_src[r] : r]); optionally dst32[r * dst32_stride] = the same row in fp32
-cudaError_t cast_rows(Launch L, int dtype, const float *src, const int32_t *row_src, void *dst,
+cudaError_t cast_rows(Launch L, int dtype, const float *src, const int32_t *row_src, Operand dst,
                       float *dst32, int dst32_stride, int R, int H);
 cudaError_t reduce_splits(Launch L, SplitIn P, float *Y, int ldy, int R, int ncols);
 
 // gemm_simt.cu : Y[R][sum n_out] (fp32, ld ldy) = X[R][K_in] * W^T, X and W of `dtype`
-cudaError_t gemm_simt(Launch L, int dtype, const void *X, GemmMats m, int K_in, int R, float *Y,
+cudaError_t gemm_simt(Launch L, int dtype, Operand X, GemmMats m, int K_in, int R, float *Y,
                       int ldy);
 
 // gemm_tc.cu : bf16 tensor-core path; writes `split` partial matrices `split_stride` apart.
 int tc_init_driver(char *err, size_t errlen);   // 0 on success
 bool tc_supported(const GemmMats &m, int K_in);
 int tc_default_split(int n_tiles, int kblocks);
-cudaError_t gemm_tc(Launch L, const void *X, int x_rows_alloc, GemmMats m, int K_in, int R,
+cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in, int R,
                     float *Y, int ldy, int split, size_t split_stride, int *status);
 
 // tree.cu

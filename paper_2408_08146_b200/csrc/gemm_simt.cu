@@ -13,7 +13,7 @@ constexpr int WARPS = 8;
 
 template <typename T>
 __global__ void __launch_bounds__(WARPS * 32)
-gemm_simt_kernel(const T *__restrict__ X, int R, int K_in, const T *__restrict__ W0,
+gemm_simt_kernel(const T *__restrict__ X, const T *__restrict__ Xlo, int R, int K_in, const T *__restrict__ W0,
                  const T *__restrict__ W1, const T *__restrict__ W2, int n0, int n1, int n2,
                  float *__restrict__ Y, int ldy) {
   __shared__ float xs[ROWS][KC + 1];
@@ -44,7 +44,13 @@ gemm_simt_kernel(const T *__restrict__ X, int R, int K_in, const T *__restrict__
     __syncthreads();
     for (int e = threadIdx.x; e < ROWS * KC; e += WARPS * 32) {
       const int r = e / KC, k = e % KC;
-      xs[r][k] = (r0 + r < R && k0 + k < K_in) ? to_f(X[(size_t)(r0 + r) * K_in + k0 + k]) : 0.f;
+      float v = 0.f;
+      if (r0 + r < R && k0 + k < K_in) {
+        const size_t idx = (size_t)(r0 + r) * K_in + k0 + k;
+        v = to_f(X[idx]);
+        if (Xlo != nullptr) v += to_f(Xlo[idx]);
+      }
+      xs[r][k] = v;
     }
     __syncthreads();
     const int kend = min(KC, K_in - k0);
@@ -71,17 +77,17 @@ gemm_simt_kernel(const T *__restrict__ X, int R, int K_in, const T *__restrict__
 
 }  // namespace
 
-cudaError_t gemm_simt(Launch L, int dtype, const void *X, GemmMats m, int K_in, int R, float *Y,
+cudaError_t gemm_simt(Launch L, int dtype, Operand X, GemmMats m, int K_in, int R, float *Y,
                       int ldy) {
   const int n0 = m.n_out[0], n1 = m.n > 1 ? m.n_out[1] : 0, n2 = m.n > 2 ? m.n_out[2] : 0;
   const int ntot = n0 + n1 + n2;
   dim3 grid((ntot + WARPS * FPW - 1) / (WARPS * FPW), (R + ROWS - 1) / ROWS);
   if (dtype == 0)
-    return launch_k(gemm_simt_kernel<float>, grid, dim3(WARPS * 32), 0, L.st, L.pdl, (const float *)X,
-                    R, K_in, (const float *)m.W[0], (const float *)(m.n > 1 ? m.W[1] : m.W[0]),
+    return launch_k(gemm_simt_kernel<float>, grid, dim3(WARPS * 32), 0, L.st, L.pdl, (const float *)X.hi,
+                    (const float *)X.lo, R, K_in, (const float *)m.W[0], (const float *)(m.n > 1 ? m.W[1] : m.W[0]),
                     (const float *)(m.n > 2 ? m.W[2] : m.W[0]), n0, n1, n2, Y, ldy);
-  return launch_k(gemm_simt_kernel<bf16>, grid, dim3(WARPS * 32), 0, L.st, L.pdl, (const bf16 *)X, R,
-                  K_in, (const bf16 *)m.W[0], (const bf16 *)(m.n > 1 ? m.W[1] : m.W[0]),
+  return launch_k(gemm_simt_kernel<bf16>, grid, dim3(WARPS * 32), 0, L.st, L.pdl, (const bf16 *)X.hi,
+                  (const bf16 *)X.lo, R, K_in, (const bf16 *)m.W[0], (const bf16 *)(m.n > 1 ? m.W[1] : m.W[0]),
                   (const bf16 *)(m.n > 2 ? m.W[2] : m.W[0]), n0, n1, n2, Y, ldy);
 }
 

@@ -10,6 +10,10 @@
 // warp 1 issues the MMAs, warps 2..5 read the accumulator back (tcgen05.ld) and store it.
 // The weight stream does not depend on the previous kernel, so under programmatic dependent
 // launch the first stages are requested before waiting for the producer of X.
+// Activations may come as a pair hi + lo of bf16 matrices (lo = rounding residual of hi): the
+// token tile then holds the hi rows followed by the lo rows of the same tokens (MMA N doubles),
+// and the epilogue adds the two halves of the accumulator, so the product carries 16 significant
+// bits of the activations at no extra weight traffic.
 // Split-K: grid.y CTAs share a weight tile and write separate partial outputs that the consumer
 // kernel sums in a fixed order (deterministic).
 // Every wait is bounded: on expiry the kernel records KOALA_E_TIMEOUT in *status, drains, frees
@@ -112,7 +116,10 @@ struct TcParams {
   float *Y;
   int ldy;
   int R;              // valid tokens
-  int bn;             // token tile (MMA N), multiple of 16, <= 256
+  int bn;             // MMA N = rows of the activation tile in shared memory, multiple of 16, <= 256
+  int tt;             // tokens per tile: bn, or bn / 2 when the activations are a hi/lo pair
+  int pair;           // 1: hi/lo pair
+  int ztiles;         // token tiles (fastest-varying part of blockIdx.x)
   int tmem_cols;      // power of two >= max(32, bn)
   int tiles0, tiles1; // weight tiles of matrix 0 and of matrices 0+1 (cumulative)
   int n0, n1, n2;     // rows of each matrix
@@ -126,7 +133,7 @@ struct TcParams {
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
                const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX,
-               const TcParams P) {
+               const __grid_constant__ CUtensorMap tmXlo, const TcParams P) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ uint64_t full_bar[MAX_STAGES];
   __shared__ uint64_t empty_bar[MAX_STAGES];
@@ -141,13 +148,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   const int stage_bytes = W_STAGE_BYTES + x_stage_bytes;   // both multiples of 1024 (bn % 16 == 0 -> x multiple of 2048)
 
   // which matrix / which rows
-  int tile = blockIdx.x;
+  int tile = blockIdx.x / P.ztiles;
+  const int ztile = blockIdx.x % P.ztiles;
   const CUtensorMap *tmW = &tmW0;
   int col_off = 0, n_rows = P.n0;
   if (tile >= P.tiles1) { tmW = &tmW2; tile -= P.tiles1; col_off = P.n0 + P.n1; n_rows = P.n2; }
   else if (tile >= P.tiles0) { tmW = &tmW1; tile -= P.tiles0; col_off = P.n0; n_rows = P.n1; }
   const int row0 = tile * BM;
-  const int tok0 = blockIdx.z * P.bn;
+  const int tok0 = ztile * P.tt;
   // K range of this split
   const int kb_lo = (int)(((long long)P.kblocks * blockIdx.y) / P.split);
   const int kb_hi = (int)(((long long)P.kblocks * (blockIdx.y + 1)) / P.split);
@@ -180,6 +188,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(tmW) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
+      if (P.pair) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmXlo) : "memory");
       const int pre = nkb < P.stages ? nkb : P.stages;
       // weights first: they do not depend on the kernel before this one
       for (int it = 0; it < pre; ++it) {
@@ -187,9 +196,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, (kb_lo + it) * BK, row0);
       }
       pdl_wait();
-      for (int it = 0; it < pre; ++it)
-        tma_load_2d(&tmX, &full_bar[it], tiles + (size_t)it * stage_bytes + W_STAGE_BYTES,
-                    (kb_lo + it) * BK, tok0);
+      const int lo_off = P.tt * BK * 2;          // the lo rows follow the hi rows of the tile
+      for (int it = 0; it < pre; ++it) {
+        unsigned char *xd = tiles + (size_t)it * stage_bytes + W_STAGE_BYTES;
+        tma_load_2d(&tmX, &full_bar[it], xd, (kb_lo + it) * BK, tok0);
+        if (P.pair) tma_load_2d(&tmXlo, &full_bar[it], xd + lo_off, (kb_lo + it) * BK, tok0);
+      }
       bool ok = true;
       for (int it = pre; it < nkb && ok; ++it) {
         const int s = it % P.stages;
@@ -200,6 +212,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         unsigned char *dst = tiles + (size_t)s * stage_bytes;
         tma_load_2d(tmW, &full_bar[s], dst, (kb_lo + it) * BK, row0);
         tma_load_2d(&tmX, &full_bar[s], dst + W_STAGE_BYTES, (kb_lo + it) * BK, tok0);
+        if (P.pair) tma_load_2d(&tmXlo, &full_bar[s], dst + W_STAGE_BYTES + lo_off, (kb_lo + it) * BK, tok0);
       }
       if (!ok) {
         atomicExch(&s_error, 1);
@@ -238,27 +251,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quarter = warp & 3;        // the 32 tensor-memory lanes this warp may read
     pdl_wait();                          // the output buffer may still be read by the previous kernel
-    bool ok = true;
-    if (nkb > 0) ok = mbar_wait(&accum_bar, 0);
+    bool ok = mbar_wait(&accum_bar, 0);
     if (!ok) atomicExch(&s_error, 1);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const int feat = row0 + quarter * 32 + lane;
     float *Yp = P.Y + (size_t)blockIdx.y * P.split_stride + col_off + feat;
     if (ok) {
-      for (int c0 = 0; c0 < P.bn; c0 += 16) {
-        uint32_t v[16];
-        if (nkb > 0) {
-          tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = 0u;
-        }
+      for (int c0 = 0; c0 < P.tt; c0 += 16) {
+        uint32_t v[16], u[16];
+        const uint32_t lane_base = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+        tmem_ld16(lane_base + (uint32_t)c0, v);
+        if (P.pair) tmem_ld16(lane_base + (uint32_t)(P.tt + c0), u);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (feat < n_rows) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int t = tok0 + c0 + j;
-            if (t < P.R) Yp[(size_t)t * P.ldy] = __uint_as_float(v[j]);
+            float r = __uint_as_float(v[j]);
+            if (P.pair) r += __uint_as_float(u[j]);
+            if (t < P.R) Yp[(size_t)t * P.ldy] = r;
           }
         }
       }
@@ -363,14 +374,24 @@ int tc_default_split(int n_tiles, int kblocks) {
   return best;
 }
 
-cudaError_t gemm_tc(Launch L, const void *X, int x_rows_alloc, GemmMats m, int K_in, int R,
+cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in, int R,
                     float *Y, int ldy, int split, size_t split_stride, int *status) {
-  if (!tc_supported(m, K_in) || R < 1) return cudaErrorInvalidValue;
+  if (!tc_supported(m, K_in) || R < 1 || ((uintptr_t)X.hi & 15u) || ((uintptr_t)X.lo & 15u))
+    return cudaErrorInvalidValue;
   TcParams P;
   memset(&P, 0, sizeof(P));
-  int bn = ((R + 15) / 16) * 16;
-  if (bn > 256) bn = 256;
-  if (bn > x_rows_alloc) return cudaErrorInvalidValue;
+  const int pair = X.lo != nullptr ? 1 : 0;
+  const int tt_max = pair ? 128 : 256;
+  int tt = ((R + 15) / 16) * 16;
+  if (tt > tt_max) tt = tt_max;
+  if (tt > x_rows_alloc) return cudaErrorInvalidValue;
+  const int bn = pair ? 2 * tt : tt;
+  const int ztiles = (R + tt - 1) / tt;
+  // the last token tile may reach past R: those rows must exist (they are read, results dropped)
+  if (ztiles * tt > x_rows_alloc) return cudaErrorInvalidValue;
+  P.tt = tt;
+  P.pair = pair;
+  P.ztiles = ztiles;
   int cols = 32;
   while (cols < bn) cols <<= 1;
   P.Y = Y;
@@ -398,15 +419,16 @@ cudaError_t gemm_tc(Launch L, const void *X, int x_rows_alloc, GemmMats m, int K
   if (stages > 8) stages = 8;
   if (stages < 2) return cudaErrorInvalidValue;
   P.stages = stages;
-  CUtensorMap mw[3], mx;
+  CUtensorMap mw[3], mx, mxlo;
   for (int i = 0; i < 3; ++i) {
     const int j = i < m.n ? i : 0;
     if (!get_map(m.W[j], m.n_out[j], K_in, BM, &mw[i])) return cudaErrorInvalidValue;
   }
-  if (!get_map(X, x_rows_alloc, K_in, bn, &mx)) return cudaErrorInvalidValue;
-  dim3 grid(t0 + t1 + t2, split, (R + bn - 1) / bn);
+  if (!get_map(X.hi, x_rows_alloc, K_in, tt, &mx)) return cudaErrorInvalidValue;
+  if (!get_map(pair ? X.lo : X.hi, x_rows_alloc, K_in, tt, &mxlo)) return cudaErrorInvalidValue;
+  dim3 grid((t0 + t1 + t2) * ztiles, split, 1);
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  return launch_k(gemm_tc_kernel, grid, dim3(THREADS), smem, L.st, L.pdl, mw[0], mw[1], mw[2], mx, P);
+  return launch_k(gemm_tc_kernel, grid, dim3(THREADS), smem, L.st, L.pdl, mw[0], mw[1], mw[2], mx, mxlo, P);
 }
 
 }  // namespace koala

@@ -13,6 +13,7 @@ using namespace koala;
 
 namespace koala {
 void tc_forget_maps();
+unsigned long long g_launches = 0;
 }
 
 namespace {
@@ -55,19 +56,27 @@ struct koala_ctx {
   size_t pcols;           // widest GEMM output
   // workspace
   float *x, *qbuf, *P, *verify_logits, *draft_logits, *verify_hid, *feat[2], *mx;
-  void *xn, *attn_out, *act, *cat, *lmin;
+  Operand xn, attn_out, act, cat, lmin;
+  bool pair;              // bf16 activations kept as hi + lo
   int32_t *verify_tgt, *s_parent, *s_level, *s_rank;
   int *status;
   TreeBufs t;
   PlanBufs p;
   // host state
   Phase phase;
-  int last_pass, pend_cap, draft_rows;
+  int last_pass, pend_cap, draft_rows, expand_mode;
   bool last_tree_from_caller;
   int *host_status;       // pinned
   cudaEvent_t poll_ev;
   bool poll_pending;
   int last_status;
+  // per-kernel timing (KOALA_OPT_TIMING)
+  bool timing;
+  std::vector<cudaEvent_t> ev;          // pairs: start, stop
+  std::vector<int> ev_cls;              // class of each pair
+  size_t ev_used;                       // pairs in use
+  uint64_t t_bytes[3];
+  int32_t t_launches[3];
   char err[256];
 };
 
@@ -142,11 +151,20 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
   c->feat[0] = w.take<float>((size_t)(B * k + 16) * H);
   c->feat[1] = w.take<float>((size_t)(B * k + 16) * H);
   c->mx = w.take<float>((size_t)Mp * H);
-  c->xn = w.take<unsigned char>((size_t)Mp * H * esz);
-  c->attn_out = w.take<unsigned char>((size_t)Mp * H * esz);
-  c->act = w.take<unsigned char>((size_t)Mp * F * esz);
-  c->cat = w.take<unsigned char>((size_t)Mp * 2 * H * esz);
-  c->lmin = w.take<unsigned char>((size_t)Mp * H * esz);
+  const bool pair = cfg.dtype == KOALA_BF16 && (cfg.flags & KOALA_F_BF16_ACTIVATIONS) == 0;
+  c->pair = pair;
+  auto operand = [&](size_t cols) {
+    Operand o;
+    o.hi = w.take<unsigned char>((size_t)Mp * cols * esz);
+    o.lo = pair ? (void *)w.take<unsigned char>((size_t)Mp * cols * esz) : nullptr;
+    if (!base) o.lo = nullptr;
+    return o;
+  };
+  c->xn = operand(H);
+  c->attn_out = operand(H);
+  c->act = operand(F);
+  c->cat = operand(2 * H);
+  c->lmin = operand(H);
   c->verify_tgt = w.take<int32_t>(Mp);
   c->s_parent = w.take<int32_t>(N);
   c->s_level = w.take<int32_t>(N);
@@ -191,28 +209,56 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
 
 Launch LN(koala_ctx *c) { return Launch{c->st, c->pdl}; }
 
+constexpr size_t MAX_TIMED = 8192;
+
+// Opens a timed bracket (returns its index, or -1 when timing is off / the pool is full).
+int time_begin(koala_ctx *c, int cls, uint64_t bytes) {
+  if (!c->timing || c->ev_used >= MAX_TIMED) return -1;
+  if (c->ev.size() < 2 * (c->ev_used + 1)) {
+    cudaEvent_t a, b;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return -1;
+    c->ev.push_back(a);
+    c->ev.push_back(b);
+    c->ev_cls.push_back(cls);
+  }
+  const int i = (int)c->ev_used++;
+  c->ev_cls[i] = cls;
+  c->t_bytes[cls] += bytes;
+  c->t_launches[cls] += 1;
+  cudaEventRecord(c->ev[2 * i], c->st);
+  return i;
+}
+void time_end(koala_ctx *c, int i) {
+  if (i >= 0) cudaEventRecord(c->ev[2 * i + 1], c->st);
+}
+
 RowPlan row_plan(koala_ctx *c) {
   return RowPlan{c->p.pos, c->p.slot, c->p.mask, c->p.ctx_len, c->p.kv_len, c->p.rope};
 }
 
 // Y = X * [W...]^T as a (possibly split) fp32 result in the partial buffer, or directly into
 // `direct` (ld = ld_direct) when given.
-int do_gemm(koala_ctx *c, const void *X, int K_in, GemmMats m, int R, float *direct, int ld_direct,
+int do_gemm(koala_ctx *c, Operand X, int K_in, GemmMats m, int R, float *direct, int ld_direct,
             SplitIn *out) {
   int ncols = 0;
   for (int i = 0; i < m.n; ++i) ncols += m.n_out[i];
   float *Y = direct ? direct : c->P;
   const int ld = direct ? ld_direct : ncols;
+  const uint64_t wbytes = (uint64_t)ncols * K_in * c->esz;
   if (c->use_tc && c->cfg.dtype == KOALA_BF16 && tc_supported(m, K_in)) {
     int tiles = 0;
     for (int i = 0; i < m.n; ++i) tiles += (m.n_out[i] + 127) / 128;
     int split = direct ? 1 : tc_default_split(tiles, K_in / 64);
     if (split > MAX_SPLIT) split = MAX_SPLIT;
     const size_t stride = (size_t)c->Mp * ld;
+    const int tb = time_begin(c, KOALA_CLS_GEMM_TC, wbytes);
     CU_TRY(gemm_tc(LN(c), X, c->Mp, m, K_in, R, Y, ld, split, stride, c->status));
+    time_end(c, tb);
     if (out) *out = SplitIn{Y, split, stride, ld};
   } else {
+    const int tb = time_begin(c, KOALA_CLS_GEMM_SIMT, wbytes);
     CU_TRY(gemm_simt(LN(c), c->cfg.dtype, X, m, K_in, R, Y, ld));
+    time_end(c, tb);
     if (out) *out = SplitIn{Y, 1, 0, ld};
   }
   return KOALA_OK;
@@ -228,7 +274,7 @@ int do_gemm(koala_ctx *c, const void *X, int K_in, GemmMats m, int R, float *dir
 // normalised input of the attention block.  On exit x is updated and `next_xn` holds
 // T(rmsnorm(x) * next_g) (or T(x) if next_g is null); `out_f32` optionally receives the same in fp32.
 int run_layer(koala_ctx *c, const LayerW &w, void *kc, void *vc, int R, int rows_per_seq,
-              const void *next_g, void *next_xn, float *out_f32) {
+              const void *next_g, Operand next_xn, float *out_f32) {
   const koala_config &g = c->cfg;
   const int H = g.H, F = g.F;
   SplitIn s;
@@ -236,8 +282,10 @@ int run_layer(koala_ctx *c, const LayerW &w, void *kc, void *vc, int R, int rows
   K_TRY(do_gemm(c, c->xn, H, qkv, R, nullptr, 0, &s));
   CU_TRY(rope_kv_write(LN(c), g.dtype, s, row_plan(c), c->qbuf, kc, vc, R, rows_per_seq, g.n_heads,
                        g.head_dim, g.S_max));
+  const int ta = time_begin(c, KOALA_CLS_ATTENTION, 0);
   CU_TRY(tree_attention(LN(c), g.dtype, c->qbuf, kc, vc, row_plan(c), c->attn_out, R, rows_per_seq, g.B,
                         g.n_heads, g.head_dim, g.S_max));
+  time_end(c, ta);
   GemmMats o{{w.wo, nullptr, nullptr}, {H, 0, 0}, 1};
   K_TRY(do_gemm(c, c->attn_out, H, o, R, nullptr, 0, &s));
   CU_TRY(row_epilogue(LN(c), g.dtype, 0, c->x, s, nullptr, w.ffn_norm, c->xn, nullptr, R, H, g.rms_eps));
@@ -276,7 +324,8 @@ int draft_eagle(koala_ctx *c, int pass) {
   // pass 0: the feature of every row stays in x and the last valid row is gathered afterwards;
   // pass >= 1: every row's feature goes to feat[pass & 1] and to the LM head's input.
   float *f_all = pass == 0 ? nullptr : c->feat[pass & 1];
-  void *lm_all = pass == 0 ? nullptr : c->lmin;
+  const Operand none{nullptr, nullptr};
+  const Operand lm_all = pass == 0 ? none : c->lmin;
   if (g.K == 0) {
     CU_TRY(row_epilogue(LN(c), g.dtype, 1, c->x, s, c->fc_b, nullptr, lm_all, f_all, R, H, g.rms_eps));
   } else {
@@ -311,7 +360,8 @@ int draft_medusa(koala_ctx *c) {
     for (int i = 0; i < nh; ++i) {
       SplitIn s;
       GemmMats m{{c->res_w[(size_t)i * g.K + j], nullptr, nullptr}, {H, 0, 0}, 1};
-      unsigned char *xi = (unsigned char *)c->xn + (size_t)i * B * H * c->esz;
+      const size_t off = (size_t)i * B * H * c->esz;
+      Operand xi{(unsigned char *)c->xn.hi + off, c->xn.lo ? (unsigned char *)c->xn.lo + off : nullptr};
       K_TRY(do_gemm(c, xi, H, m, B, nullptr, 0, &s));
       CU_TRY(row_epilogue(LN(c), g.dtype, 2, c->mx + (size_t)i * B * H, s, c->res_b[(size_t)i * g.K + j],
                           nullptr, xi, nullptr, B, H, g.rms_eps));
@@ -426,6 +476,11 @@ int koala_init(const koala_config *cfg, const koala_weights *w, const koala_stat
   c->last_pass = -1;
   c->pend_cap = g.N < g.D + 1 ? g.N : g.D + 1;
   c->draft_rows = 0;
+  c->expand_mode = 0;
+  c->timing = false;
+  c->ev_used = 0;
+  memset(c->t_bytes, 0, sizeof(c->t_bytes));
+  memset(c->t_launches, 0, sizeof(c->t_launches));
   c->last_tree_from_caller = false;
   return KOALA_OK;
 }
@@ -455,7 +510,9 @@ int koala_expand_tree(koala_ctx *c, int pass) {
   const koala_config &g = c->cfg;
   if (c->phase != PH_DRAFTED || c->last_pass != pass)
     return fail(c, KOALA_E_STATE, "koala_expand_tree(%d) must follow koala_draft(%d)", pass, pass);
-  CU_TRY(topk_logp(LN(c), c->draft_logits, c->t.topk_tok, c->t.topk_logp, c->draft_rows, g.V, g.topk));
+  if (c->expand_mode != 2)
+    CU_TRY(topk_logp(LN(c), c->draft_logits, c->t.topk_tok, c->t.topk_logp, c->draft_rows, g.V, g.topk));
+  if (c->expand_mode == 1) return KOALA_OK;
   if (g.head_kind == KOALA_MEDUSA) {
     CU_TRY(expand_static(LN(c), c->t, c->s_parent, c->s_level, c->s_rank, g.B, g.N, g.topk));
     c->phase = PH_TREE;
@@ -545,6 +602,40 @@ int koala_buffers(koala_ctx *c, koala_buffer_table *o) {
   return KOALA_OK;
 }
 
+int koala_set_option(koala_ctx *c, int option, int value) {
+  if (!c) return KOALA_E_INVALID;
+  if (option == KOALA_OPT_EXPAND_MODE && value >= 0 && value <= 2) {
+    c->expand_mode = value;
+    return KOALA_OK;
+  }
+  if (option == KOALA_OPT_TIMING && (value == 0 || value == 1)) {
+    c->timing = value == 1;
+    c->ev_used = 0;
+    memset(c->t_bytes, 0, sizeof(c->t_bytes));
+    memset(c->t_launches, 0, sizeof(c->t_launches));
+    return KOALA_OK;
+  }
+  return fail(c, KOALA_E_INVALID, "unknown option %d / value %d", option, value);
+}
+
+int koala_timing_read(koala_ctx *c, koala_timing *out) {
+  if (!c || !out) return KOALA_E_INVALID;
+  memset(out, 0, sizeof(*out));
+  CU_TRY(cudaStreamSynchronize(c->st));
+  for (size_t i = 0; i < c->ev_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->ev[2 * i], c->ev[2 * i + 1]) == cudaSuccess) out->ms[c->ev_cls[i]] += ms;
+  }
+  for (int k = 0; k < 3; ++k) {
+    out->bytes[k] = c->t_bytes[k];
+    out->launches[k] = c->t_launches[k];
+  }
+  (void)cudaGetLastError();
+  return KOALA_OK;
+}
+
+uint64_t koala_launch_count(void) { return (uint64_t)koala::g_launches; }
+
 int koala_poll(koala_ctx *c, int *done, int *device_status) {
   if (!c) return KOALA_E_INVALID;
   if (c->poll_pending && cudaEventQuery(c->poll_ev) == cudaSuccess) {
@@ -572,8 +663,17 @@ void koala_destroy(koala_ctx *c) {
   if (!c) return;
   if (c->host_status) cudaFreeHost(c->host_status);
   if (c->poll_ev) cudaEventDestroy(c->poll_ev);
+  for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
   koala::tc_forget_maps();
   delete c;
+}
+
+int koala_gemm_x_rows(int M, int has_lo) {
+  if (M < 1) return 0;
+  const int tt_max = has_lo ? 128 : 256;
+  int tt = (M + 15) / 16 * 16;
+  if (tt > tt_max) tt = tt_max;
+  return (M + tt - 1) / tt * tt;
 }
 
 size_t koala_gemm_scratch_bytes(int M, int N_out, int K_in) {
@@ -582,13 +682,14 @@ size_t koala_gemm_scratch_bytes(int M, int N_out, int K_in) {
   return (size_t)MAX_SPLIT * ((size_t)M + 16) * (size_t)N_out * sizeof(float);
 }
 
-int koala_gemm_bf16(const void *X, const void *W, float *Y, int ldy, int M, int N_out, int K_in,
+int koala_gemm_bf16(const void *X, const void *X_lo, const void *W, float *Y, int ldy, int M, int N_out, int K_in,
                     void *scratch, size_t scratch_bytes, int use_tensor_cores, int split_k,
                     void *cuda_stream, int *device_status) {
   if (!X || !W || !Y || M < 1 || N_out < 1 || K_in < 1 || ldy < N_out) return KOALA_E_INVALID;
   Launch L{(cudaStream_t)cuda_stream, false};
   GemmMats m{{W, nullptr, nullptr}, {N_out, 0, 0}, 1};
-  if (!use_tensor_cores) return gemm_simt(L, KOALA_BF16, X, m, K_in, M, Y, ldy) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
+  Operand Xo{const_cast<void *>(X), const_cast<void *>(X_lo)};
+  if (!use_tensor_cores) return gemm_simt(L, KOALA_BF16, Xo, m, K_in, M, Y, ldy) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
   char e[160];
   if (tc_init_driver(e, sizeof(e)) != 0) return KOALA_E_CUDA;
   if (!tc_supported(m, K_in)) return KOALA_E_UNSUPPORTED;
@@ -597,13 +698,13 @@ int koala_gemm_bf16(const void *X, const void *W, float *Y, int ldy, int M, int 
   if (split > K_in / 64) split = K_in / 64;
   // X must hold a whole token tile: the caller's buffer has M rows, rounded up by the map's
   // out-of-bounds zero fill
-  const int rows_alloc = ((M + 15) / 16) * 16;
+  const int rows_alloc = koala_gemm_x_rows(M, X_lo != nullptr);
   if (split == 1) {
-    return gemm_tc(L, X, rows_alloc, m, K_in, M, Y, ldy, 1, 0, device_status) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
+    return gemm_tc(L, Xo, rows_alloc, m, K_in, M, Y, ldy, 1, 0, device_status) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
   }
   const size_t stride = (size_t)M * N_out;
   if (!scratch || scratch_bytes < (size_t)split * stride * sizeof(float)) return KOALA_E_CAPACITY;
-  if (gemm_tc(L, X, rows_alloc, m, K_in, M, (float *)scratch, N_out, split, stride, device_status) != cudaSuccess)
+  if (gemm_tc(L, Xo, rows_alloc, m, K_in, M, (float *)scratch, N_out, split, stride, device_status) != cudaSuccess)
     return KOALA_E_CUDA;
   SplitIn s{(const float *)scratch, split, stride, N_out};
   return reduce_splits(L, s, Y, ldy, M, N_out) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;

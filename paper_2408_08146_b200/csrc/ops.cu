@@ -25,11 +25,21 @@ __device__ __forceinline__ float block_sum(float v, float *red) {
 
 __device__ __forceinline__ float silu_f(float v) { return v / (1.f + expf(-v)); }
 
+// Stores v as a matrix-multiply operand.  bf16 operands are kept as a pair hi + lo (lo = the
+// rounding residual of hi, itself rounded to bf16), which carries 16 significant bits into the
+// tensor cores; fp32 operands are exact and have no lo part.
+template <typename T>
+__device__ __forceinline__ void store_operand(T *hi, T *lo, size_t i, float v) {
+  const T h = from_f<T>(v);
+  hi[i] = h;
+  if (lo != nullptr) lo[i] = from_f<T>(v - to_f(h));
+}
+
 // ------------------------------------------------------------------------------- embedding + norm
 template <typename T>
 __global__ void embed_norm_kernel(const int32_t *__restrict__ tok, const T *__restrict__ E,
                                   const T *__restrict__ g, float *__restrict__ x,
-                                  T *__restrict__ xn, int H, int V, float eps) {
+                                  T *__restrict__ xn, T *__restrict__ xn_lo, int H, int V, float eps) {
   __shared__ float red[32];
   pdl_launch_dependents();
   pdl_wait();
@@ -45,15 +55,15 @@ __global__ void embed_norm_kernel(const int32_t *__restrict__ tok, const T *__re
   }
   const float inv = rsqrtf(block_sum(ss, red) / (float)H + eps);
   for (int i = threadIdx.x; i < H; i += blockDim.x)
-    xn[(size_t)r * H + i] = from_f<T>(x[(size_t)r * H + i] * inv * to_f(g[i]));
+    store_operand(xn, xn_lo, (size_t)r * H + i, x[(size_t)r * H + i] * inv * to_f(g[i]));
 }
 
 // ------------------------------------------------------------------------------- row epilogue
 template <typename T>
 __global__ void row_epilogue_kernel(int mode, float *__restrict__ x, SplitIn P,
                                     const T *__restrict__ bias, const T *__restrict__ g,
-                                    T *__restrict__ xn, float *__restrict__ out_f32, int H,
-                                    float eps) {
+                                    T *__restrict__ xn, T *__restrict__ xn_lo,
+                                    float *__restrict__ out_f32, int H, float eps) {
   __shared__ float red[32];
   pdl_launch_dependents();
   pdl_wait();
@@ -74,7 +84,7 @@ __global__ void row_epilogue_kernel(int mode, float *__restrict__ x, SplitIn P,
   for (int i = threadIdx.x; i < H; i += blockDim.x) {
     float n = xr[i];
     if (g != nullptr) n = n * inv * to_f(g[i]);
-    if (xn != nullptr) xn[(size_t)r * H + i] = from_f<T>(n);
+    if (xn != nullptr) store_operand(xn, xn_lo, (size_t)r * H + i, n);
     if (out_f32 != nullptr) out_f32[(size_t)r * H + i] = n;
   }
 }
@@ -84,7 +94,7 @@ template <typename T>
 __global__ void eagle_concat_kernel(const float *__restrict__ feat_src,
                                     const int32_t *__restrict__ row_src,
                                     const int32_t *__restrict__ row_tok, const T *__restrict__ E,
-                                    T *__restrict__ cat, int H, int V) {
+                                    T *__restrict__ cat, T *__restrict__ cat_lo, int H, int V) {
   pdl_launch_dependents();
   pdl_wait();
   const int r = blockIdx.x;
@@ -93,24 +103,25 @@ __global__ void eagle_concat_kernel(const float *__restrict__ feat_src,
   t = t < 0 ? 0 : (t >= V ? V - 1 : t);
   const float *f = feat_src + (size_t)src * H;
   const T *e = E + (size_t)t * H;
-  T *c = cat + (size_t)r * 2 * H;
+  const size_t base = (size_t)r * 2 * H;
   for (int i = threadIdx.x; i < H; i += blockDim.x) {
-    c[i] = from_f<T>(f[i]);
-    c[H + i] = e[i];
+    store_operand(cat, cat_lo, base + i, f[i]);
+    cat[base + H + i] = e[i];
+    if (cat_lo != nullptr) cat_lo[base + H + i] = from_f<T>(0.f);
   }
 }
 
 template <typename T>
 __global__ void cast_rows_kernel(const float *__restrict__ src, const int32_t *__restrict__ row_src,
-                                 T *__restrict__ dst, float *__restrict__ dst32, int dst32_stride,
-                                 int H) {
+                                 T *__restrict__ dst, T *__restrict__ dst_lo,
+                                 float *__restrict__ dst32, int dst32_stride, int H) {
   pdl_launch_dependents();
   pdl_wait();
   const int r = blockIdx.x;
   const int s = row_src ? row_src[r] : r;
   for (int i = threadIdx.x; i < H; i += blockDim.x) {
     const float v = src[(size_t)s * H + i];
-    dst[(size_t)r * H + i] = from_f<T>(v);
+    store_operand(dst, dst_lo, (size_t)r * H + i, v);
     if (dst32) dst32[(size_t)r * dst32_stride * H + i] = v;
   }
 }
@@ -152,13 +163,13 @@ __global__ void rope_kv_kernel(SplitIn qkv, RowPlan plan, float *__restrict__ q_
 
 // ------------------------------------------------------------------------------- SwiGLU
 template <typename T>
-__global__ void swiglu_kernel(SplitIn gu, T *__restrict__ act, int F) {
+__global__ void swiglu_kernel(SplitIn gu, T *__restrict__ act, T *__restrict__ act_lo, int F) {
   pdl_launch_dependents();
   pdl_wait();
   const int r = blockIdx.y;
   const int f = blockIdx.x * blockDim.x + threadIdx.x;
   if (f >= F) return;
-  act[(size_t)r * F + f] = from_f<T>(silu_f(gu.at(r, f)) * gu.at(r, F + f));
+  store_operand(act, act_lo, (size_t)r * F + f, silu_f(gu.at(r, f)) * gu.at(r, F + f));
 }
 
 // ------------------------------------------------------------------------------- tree attention
@@ -168,7 +179,8 @@ __global__ void swiglu_kernel(SplitIn gu, T *__restrict__ act, int F) {
 template <typename T, int DH>
 __global__ void __launch_bounds__(256)
 tree_attn_kernel(const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc,
-                 RowPlan plan, T *__restrict__ out, int rows_per_seq, int n_heads, int S_max) {
+                 RowPlan plan, T *__restrict__ out, T *__restrict__ out_lo, int rows_per_seq,
+                 int n_heads, int S_max) {
   __shared__ float Ks[32][DH + 1];
   __shared__ float Vs[32][DH];
   __shared__ float qs[8][DH];
@@ -227,7 +239,7 @@ tree_attn_kernel(const float *__restrict__ q, const T *__restrict__ kc, const T 
     const float inv = l > 0.f ? 1.f / l : 0.f;
 #pragma unroll
     for (int d = 0; d < DH / 32; ++d)
-      out[(size_t)r * H + h * DH + lane + 32 * d] = from_f<T>(o[d] * inv);
+      store_operand(out, out_lo, (size_t)r * H + h * DH + lane + 32 * d, o[d] * inv);
   }
 }
 
@@ -326,27 +338,29 @@ __global__ void topk_logp_kernel(const float *__restrict__ logits, int32_t *__re
   }
 
 cudaError_t embed_norm(Launch L, int dtype, const int32_t *tok, const void *E, const void *g,
-                       float *x, void *xn, int R, int H, int V, float eps) {
+                       float *x, Operand xn, int R, int H, int V, float eps) {
   DISPATCH_T(dtype, return launch_k(embed_norm_kernel<T>, dim3(R), dim3(256), 0, L.st, L.pdl, tok,
-                                    (const T *)E, (const T *)g, x, (T *)xn, H, V, eps);)
+                                    (const T *)E, (const T *)g, x, (T *)xn.hi, (T *)xn.lo, H, V, eps);)
 }
 
 cudaError_t row_epilogue(Launch L, int dtype, int mode, float *x, SplitIn P, const void *bias,
-                         const void *g, void *xn, float *out_f32, int R, int H, float eps) {
+                         const void *g, Operand xn, float *out_f32, int R, int H, float eps) {
   DISPATCH_T(dtype, return launch_k(row_epilogue_kernel<T>, dim3(R), dim3(256), 0, L.st, L.pdl, mode,
-                                    x, P, (const T *)bias, (const T *)g, (T *)xn, out_f32, H, eps);)
+                                    x, P, (const T *)bias, (const T *)g, (T *)xn.hi, (T *)xn.lo, out_f32,
+                                    H, eps);)
 }
 
 cudaError_t eagle_concat(Launch L, int dtype, const float *feat_src, const int32_t *row_src,
-                         const int32_t *row_tok, const void *E, void *cat, int R, int H, int V) {
+                         const int32_t *row_tok, const void *E, Operand cat, int R, int H, int V) {
   DISPATCH_T(dtype, return launch_k(eagle_concat_kernel<T>, dim3(R), dim3(256), 0, L.st, L.pdl,
-                                    feat_src, row_src, row_tok, (const T *)E, (T *)cat, H, V);)
+                                    feat_src, row_src, row_tok, (const T *)E, (T *)cat.hi, (T *)cat.lo, H,
+                                    V);)
 }
 
-cudaError_t cast_rows(Launch L, int dtype, const float *src, const int32_t *row_src, void *dst,
+cudaError_t cast_rows(Launch L, int dtype, const float *src, const int32_t *row_src, Operand dst,
                       float *dst32, int dst32_stride, int R, int H) {
   DISPATCH_T(dtype, return launch_k(cast_rows_kernel<T>, dim3(R), dim3(256), 0, L.st, L.pdl, src,
-                                    row_src, (T *)dst, dst32, dst32_stride, H);)
+                                    row_src, (T *)dst.hi, (T *)dst.lo, dst32, dst32_stride, H);)
 }
 
 cudaError_t reduce_splits(Launch L, SplitIn P, float *Y, int ldy, int R, int ncols) {
@@ -362,24 +376,24 @@ cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowPlan plan, float 
                                     rows_per_seq, n_heads, head_dim, S_max);)
 }
 
-cudaError_t swiglu(Launch L, int dtype, SplitIn gu, void *act, int R, int F) {
+cudaError_t swiglu(Launch L, int dtype, SplitIn gu, Operand act, int R, int F) {
   DISPATCH_T(dtype, return launch_k(swiglu_kernel<T>, dim3((F + 255) / 256, R), dim3(256), 0, L.st,
-                                    L.pdl, gu, (T *)act, F);)
+                                    L.pdl, gu, (T *)act.hi, (T *)act.lo, F);)
 }
 
 cudaError_t tree_attention(Launch L, int dtype, const float *q, const void *k_cache,
-                           const void *v_cache, RowPlan plan, void *out, int R, int rows_per_seq,
+                           const void *v_cache, RowPlan plan, Operand out, int R, int rows_per_seq,
                            int B, int n_heads, int head_dim, int S_max) {
   (void)R;
   dim3 grid((rows_per_seq + 7) / 8, n_heads, B);
   if (head_dim == 64) {
     DISPATCH_T(dtype, return launch_k(tree_attn_kernel<T, 64>, grid, dim3(256), 0, L.st, L.pdl, q,
-                                      (const T *)k_cache, (const T *)v_cache, plan, (T *)out,
-                                      rows_per_seq, n_heads, S_max);)
+                                      (const T *)k_cache, (const T *)v_cache, plan, (T *)out.hi,
+                                      (T *)out.lo, rows_per_seq, n_heads, S_max);)
   } else if (head_dim == 128) {
     DISPATCH_T(dtype, return launch_k(tree_attn_kernel<T, 128>, grid, dim3(256), 0, L.st, L.pdl, q,
-                                      (const T *)k_cache, (const T *)v_cache, plan, (T *)out,
-                                      rows_per_seq, n_heads, S_max);)
+                                      (const T *)k_cache, (const T *)v_cache, plan, (T *)out.hi,
+                                      (T *)out.lo, rows_per_seq, n_heads, S_max);)
   }
   return cudaErrorInvalidValue;
 }

@@ -2,7 +2,7 @@
 import numpy as np
 import torch
 
-from oracle.koala_oracle import KoalaOracle
+from oracle.koala_oracle import KoalaOracle, round_to_bf16
 from paper_2408_08146_b200 import Koala
 from tests.helpers import HostWeights
 from workloads.generate import WeightStore, medusa_static_tree
@@ -31,7 +31,8 @@ def make_pair(cfg, flags=0, oracle_dtype=np.float64, cache_host=True):
     st = static_tree_for(cfg)
     eng = Koala(cfg, store.tensors, static_tree=st, flags=flags)
     getter = HostWeights(store, oracle_dtype) if cache_host else StreamedWeights(store, oracle_dtype)
-    orc = KoalaOracle(cfg, getter, dtype=oracle_dtype, static_tree=st)
+    orc = KoalaOracle(cfg, getter, dtype=oracle_dtype, static_tree=st,
+                      kv_round=round_to_bf16 if cfg.dtype == 1 else None)
     return eng, orc, store
 
 

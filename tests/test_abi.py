@@ -55,4 +55,4 @@ def test_init_rejects_bad_arguments_before_touching_the_device():
     assert rc == 1 and b"missing target weights" in lib.koala_last_error(ctx)
     lib.koala_destroy(ctx)
     assert lib.koala_draft(None, 0) == 1 and lib.koala_verify(None, None) == 1
-    assert lib.koala_gemm_bf16(None, None, None, 0, 0, 0, 0, None, 0, 1, 0, None, None) == 1
+    assert lib.koala_gemm_bf16(None, None, None, None, 0, 0, 0, 0, None, 0, 1, 0, None, None) == 1

@@ -43,3 +43,27 @@ def test_cuda_core_gemm(shape):
     torch.cuda.synchronize()
     err = np.abs(y.cpu().numpy() - ref).max()
     assert err <= 2e-5 * np.sqrt(K) + 1e-6, f"max err {err}"
+
+
+@pytest.mark.parametrize("shape", [(10, 4096, 4096), (60, 1536, 4096), (100, 256, 11008), (130, 384, 512),
+                                   (256, 256, 1024)])
+@pytest.mark.parametrize("tc", [True, False], ids=["tensor_core", "cuda_core"])
+def test_gemm_with_activation_pairs(shape, tc):
+    """fp32 activations given as a bf16 value + bf16 rounding residual: the product must be that of
+    the pair's sum (about 16 significant bits of the activations)."""
+    M, N, K = shape
+    xf = normal_tensor(9, f"xf{M}.{N}.{K}", (M, K), 1.0, 0.0, torch.float32, "cuda:0")
+    w = normal_tensor(8, f"w{M}.{N}.{K}", (N, K), 0.02, 0.0, torch.bfloat16, "cuda:0")
+    hi = xf.to(torch.bfloat16)
+    lo = (xf - hi.float()).to(torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    y = koala_gemm_bf16(hi, w, tc, 0, status, x_lo=lo)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref_pair = (hi.double() + lo.double()).cpu().numpy() @ w.double().cpu().numpy().T
+    ref_full = xf.double().cpu().numpy() @ w.double().cpu().numpy().T
+    assert np.abs(y.cpu().numpy() - ref_pair).max() <= 2e-5 * np.sqrt(K) + 1e-6
+    # and the pair is a much better stand-in for the fp32 activations than plain bf16
+    err_pair = np.abs(y.cpu().numpy() - ref_full).max()
+    err_bf16 = np.abs(hi.double().cpu().numpy() @ w.double().cpu().numpy().T - ref_full).max()
+    assert err_pair < 0.05 * err_bf16 + 1e-5

@@ -3,8 +3,8 @@ import itertools
 
 import numpy as np
 
-from oracle.koala_oracle import (argmax_first, log_softmax, masked_softmax, rmsnorm, rope, silu,
-                                 top_k)
+from oracle.koala_oracle import (argmax_first, log_softmax, masked_softmax, rmsnorm, rope,
+                                 round_to_bf16, silu, top_k)
 
 RNG = np.random.default_rng(11)
 
@@ -71,3 +71,16 @@ def test_top_k_against_brute_force_with_ties():
             rest.remove(i)
         assert got == want
     assert argmax_first(np.asarray([1.0, 5.0, 5.0, 2.0])) == 1
+
+
+def test_bf16_storage_rounding_matches_the_library_conversion():
+    import torch
+    x = (RNG.standard_normal(200000) * np.exp(RNG.uniform(-20, 20, 200000))).astype(np.float32)
+    # exact ties (low 16 bits = 0x8000) round to even
+    ties = (RNG.integers(0x3F00, 0x4100, 1000).astype(np.uint32) << np.uint32(16)) | np.uint32(0x8000)
+    x = np.concatenate([x, ties.view(np.float32), np.asarray([0.0, -0.0, 1.0, -1.0, 3.140625], np.float32)])
+    want = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    got = round_to_bf16(x)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    assert round_to_bf16(np.asarray([1.00390625], np.float32))[0] == 1.0          # 1 + 2^-8: tie -> even
+    assert round_to_bf16(np.asarray([1.01171875], np.float32))[0] == 1.015625     # 1 + 3*2^-8: tie -> even
