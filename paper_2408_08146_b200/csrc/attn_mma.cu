@@ -1,0 +1,320 @@
+// Tree-masked flash-decode attention for bf16 caches with head_dim 128, on tensor cores.
+//
+// One CTA = one (key chunk, head, sequence); it serves all query rows of the sequence (up to 128,
+// 16 per warp).  The sequence's keys are cut into `chunks` ranges of whole 64-key tiles from the
+// device-side length, so the grid is fixed by host-known sizes while the work follows the real
+// context length.  K and V tiles stream through shared memory with cp.async (double buffered,
+// 16-byte vector loads, XOR-swizzled rows); scores S = Q K^T and the update O += P V run on
+// mma.sync m16n8k16 with fp32 accumulators.  Q and P enter the MMAs as bf16 pairs (value +
+// rounding residual), so only the cached K and V carry bf16 rounding.  The mask is: slots below
+// ctx_len visible to every row; slot ctx_len + j visible to a row iff bit j of its 128-bit mask.
+// Softmax is online, in fp32, in base 2; row statistics use quad shuffles.  Each CTA writes an
+// unnormalised partial (O, m, l) per row; a second kernel combines the chunks in a fixed order
+// and emits the normalised output as a matrix-multiply operand.
+#include "common.cuh"
+
+namespace koala {
+namespace {
+
+constexpr int DH = 128;
+constexpr int TILE = 64;                 // keys per shared-memory tile
+constexpr int ROW_BYTES = DH * 2;        // 256
+constexpr int TILE_BYTES = TILE * ROW_BYTES;
+constexpr int PSTRIDE = DH + 2;          // floats per partial: O[128], m, l
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// byte offset of 16-byte chunk `ch` (0..15) of row `row` inside a swizzled tile
+__device__ __forceinline__ uint32_t tile_off(int row, int ch) {
+  return (uint32_t)(row * ROW_BYTES + ((ch ^ (row & 7)) << 4));
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
+  const int sz = valid ? 16 : 0;          // zero-fill when out of range
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float *d, const uint32_t *a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// two floats -> packed bf16x2 (hi) and the packed residuals (lo)
+__device__ __forceinline__ void split_pack(float x, float y, uint32_t &hi, uint32_t &lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+  const float2 hf = __bfloat1622float2(h);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(x - hf.x, y - hf.y);
+  hi = *reinterpret_cast<const uint32_t *>(&h);
+  lo = *reinterpret_cast<const uint32_t *>(&l);
+}
+
+__device__ __forceinline__ bool mask_bit(uint64_t m0, uint64_t m1, int rel) {
+  return rel < 64 ? ((m0 >> rel) & 1ull) : (rel < 128 ? ((m1 >> (rel - 64)) & 1ull) : false);
+}
+
+// grid (chunks, n_heads, B); block = max(4, compute warps) * 32 threads
+__global__ void __launch_bounds__(256)
+tree_attn_mma_kernel(const float *__restrict__ q, const bf16 *__restrict__ kc, const bf16 *__restrict__ vc,
+                     RowPlan plan, float *__restrict__ part, int rows_per_seq, int n_heads, int S_max,
+                     int chunks, int compute_warps) {
+  extern __shared__ __align__(1024) unsigned char smem[];     // [2 buffers][K tile | V tile]
+  pdl_launch_dependents();
+  pdl_wait();
+  const int c = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int H = n_heads * DH;
+  const int ctx = plan.ctx_len[b];
+  int kv_len = plan.kv_len[b];
+  kv_len = kv_len > S_max ? S_max : kv_len;
+  const int n_tiles = (kv_len + TILE - 1) / TILE;
+  const int tile_lo = (int)(((long long)n_tiles * c) / chunks);
+  const int tile_hi = (int)(((long long)n_tiles * (c + 1)) / chunks);
+  const bf16 *kb = kc + ((size_t)b * n_heads + h) * S_max * DH;
+  const bf16 *vb = vc + ((size_t)b * n_heads + h) * S_max * DH;
+  const uint32_t sbase = smem_addr(smem);
+
+  auto load_tile = [&](int tile, int buf) {
+    const int key0 = tile * TILE;
+    const uint32_t kdst = sbase + buf * 2 * TILE_BYTES, vdst = kdst + TILE_BYTES;
+    for (int e = threadIdx.x; e < TILE * 16; e += blockDim.x) {
+      const int row = e >> 4, ch = e & 15;
+      const bool in = key0 + row < kv_len;
+      const size_t goff = (size_t)(in ? key0 + row : 0) * DH + ch * 8;
+      cp_async16(kdst + tile_off(row, ch), kb + goff, in);
+      cp_async16(vdst + tile_off(row, ch), vb + goff, in);
+    }
+  };
+
+  const bool compute = warp < compute_warps;
+  // rows of this warp: i0 = warp*16 + g and i0 + 8
+  const int i0 = warp * 16 + g, i1 = i0 + 8;
+  const bool in0 = compute && i0 < rows_per_seq, in1 = compute && i1 < rows_per_seq;
+  const int r0 = b * rows_per_seq + (in0 ? i0 : 0), r1 = b * rows_per_seq + (in1 ? i1 : 0);
+  const bool ok0 = in0 && plan.slot[r0] >= 0, ok1 = in1 && plan.slot[r1] >= 0;
+  const uint64_t m00 = ok0 ? plan.mask[(size_t)r0 * 2] : 0ull, m01 = ok0 ? plan.mask[(size_t)r0 * 2 + 1] : 0ull;
+  const uint64_t m10 = ok1 ? plan.mask[(size_t)r1 * 2] : 0ull, m11 = ok1 ? plan.mask[(size_t)r1 * 2 + 1] : 0ull;
+
+  if (tile_lo < tile_hi) load_tile(tile_lo, 0);
+  cp_async_commit();
+
+  // Q fragments (A operand, 8 k-steps of 16), as bf16 pairs
+  uint32_t qh[8][4], ql[8][4];
+  if (compute) {
+    const float *q0 = q + (size_t)r0 * H + h * DH, *q1 = q + (size_t)r1 * H + h * DH;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      const int col = ks * 16 + 2 * t;
+      const float2 a = ok0 ? *reinterpret_cast<const float2 *>(q0 + col) : make_float2(0.f, 0.f);
+      const float2 bq = ok1 ? *reinterpret_cast<const float2 *>(q1 + col) : make_float2(0.f, 0.f);
+      const float2 cq = ok0 ? *reinterpret_cast<const float2 *>(q0 + col + 8) : make_float2(0.f, 0.f);
+      const float2 dq = ok1 ? *reinterpret_cast<const float2 *>(q1 + col + 8) : make_float2(0.f, 0.f);
+      split_pack(a.x, a.y, qh[ks][0], ql[ks][0]);
+      split_pack(bq.x, bq.y, qh[ks][1], ql[ks][1]);
+      split_pack(cq.x, cq.y, qh[ks][2], ql[ks][2]);
+      split_pack(dq.x, dq.y, qh[ks][3], ql[ks][3]);
+    }
+  }
+
+  float o[16][4];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+  float mrow0 = -INFINITY, mrow1 = -INFINITY, lrow0 = 0.f, lrow1 = 0.f;
+  const float sc = 0.08838834764831845f * 1.4426950408889634f;    // 1/sqrt(128) * log2(e)
+
+  for (int tile = tile_lo; tile < tile_hi; ++tile) {
+    const int buf = (tile - tile_lo) & 1;
+    if (tile + 1 < tile_hi) load_tile(tile + 1, buf ^ 1);
+    cp_async_commit();
+    cp_async_wait<1>();
+    __syncthreads();
+    if (compute) {
+      const uint32_t kt = sbase + buf * 2 * TILE_BYTES, vt = kt + TILE_BYTES;
+      const int key0 = tile * TILE;
+      // ---- S = Q K^T : 8 key groups of 8, 8 k-steps over head_dim
+      float s[8][4];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+#pragma unroll
+        for (int kp = 0; kp < 4; ++kp) {          // pairs of k-steps: 32 head dims = 4 chunks
+          uint32_t b0, b1, b2, b3;
+          ldmatrix_x4(kt + tile_off(8 * j + (lane & 7), 4 * kp + (lane >> 3)), b0, b1, b2, b3);
+          mma_bf16(s[j], qh[2 * kp], b0, b1);
+          mma_bf16(s[j], ql[2 * kp], b0, b1);
+          mma_bf16(s[j], qh[2 * kp + 1], b2, b3);
+          mma_bf16(s[j], ql[2 * kp + 1], b2, b3);
+        }
+      }
+      // ---- mask, online softmax (base 2)
+      const bool need_mask = key0 + TILE > ctx;     // tile reaches into the per-row region or past the end
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int key = key0 + 8 * j + 2 * t + e;
+          bool v0 = ok0, v1 = ok1;
+          if (need_mask) {
+            if (key >= kv_len) { v0 = false; v1 = false; }
+            else if (key >= ctx) {
+              v0 = v0 && mask_bit(m00, m01, key - ctx);
+              v1 = v1 && mask_bit(m10, m11, key - ctx);
+            }
+          }
+          s[j][e] = v0 ? s[j][e] * sc : -INFINITY;
+          s[j][2 + e] = v1 ? s[j][2 + e] * sc : -INFINITY;
+          mx0 = fmaxf(mx0, s[j][e]);
+          mx1 = fmaxf(mx1, s[j][2 + e]);
+        }
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      const float mn0 = fmaxf(mrow0, mx0), mn1 = fmaxf(mrow1, mx1);
+      const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
+      const float cr0 = exp2f(mrow0 - mu0), cr1 = exp2f(mrow1 - mu1);   // exp2(-inf) = 0
+      mrow0 = mn0;
+      mrow1 = mn1;
+      float ps0 = 0.f, ps1 = 0.f;
+      uint32_t ph[4][4], pl[4][4];       // P as A operand: 4 k-steps of 16 keys
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float p00 = exp2f(s[j][0] - mu0), p01 = exp2f(s[j][1] - mu0);
+        const float p10 = exp2f(s[j][2] - mu1), p11 = exp2f(s[j][3] - mu1);
+        ps0 += p00 + p01;
+        ps1 += p10 + p11;
+        const int ks = j >> 1, half = (j & 1) * 2;
+        split_pack(p00, p01, ph[ks][half], pl[ks][half]);
+        split_pack(p10, p11, ph[ks][half + 1], pl[ks][half + 1]);
+      }
+      ps0 += __shfl_xor_sync(0xffffffffu, ps0, 1);
+      ps0 += __shfl_xor_sync(0xffffffffu, ps0, 2);
+      ps1 += __shfl_xor_sync(0xffffffffu, ps1, 1);
+      ps1 += __shfl_xor_sync(0xffffffffu, ps1, 2);
+      lrow0 = lrow0 * cr0 + ps0;
+      lrow1 = lrow1 * cr1 + ps1;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        o[j][0] *= cr0; o[j][1] *= cr0; o[j][2] *= cr1; o[j][3] *= cr1;
+      }
+      // ---- O += P V : 4 k-steps of 16 keys, 16 groups of 8 head dims
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+        for (int jp = 0; jp < 8; ++jp) {           // pairs of head-dim groups
+          uint32_t b0, b1, b2, b3;
+          ldmatrix_x4_trans(vt + tile_off(16 * ks + (lane & 7) + 8 * ((lane >> 3) & 1), 2 * jp + (lane >> 4)),
+                            b0, b1, b2, b3);
+          mma_bf16(o[2 * jp], ph[ks], b0, b1);
+          mma_bf16(o[2 * jp], pl[ks], b0, b1);
+          mma_bf16(o[2 * jp + 1], ph[ks], b2, b3);
+          mma_bf16(o[2 * jp + 1], pl[ks], b2, b3);
+        }
+      }
+    }
+    __syncthreads();      // the buffer being refilled next iteration is no longer read
+  }
+  cp_async_wait<0>();
+  if (!compute) return;
+  // ---- partial results
+  if (in0) {
+    float *p = part + (((size_t)r0 * n_heads + h) * chunks + c) * PSTRIDE;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) *reinterpret_cast<float2 *>(p + 8 * j + 2 * t) = make_float2(o[j][0], o[j][1]);
+    if (t == 0) { p[DH] = mrow0; p[DH + 1] = lrow0; }
+  }
+  if (in1) {
+    float *p = part + (((size_t)r1 * n_heads + h) * chunks + c) * PSTRIDE;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) *reinterpret_cast<float2 *>(p + 8 * j + 2 * t) = make_float2(o[j][2], o[j][3]);
+    if (t == 0) { p[DH] = mrow1; p[DH + 1] = lrow1; }
+  }
+}
+
+// One warp per (row, head): merges the chunk partials in chunk order and writes the operand pair.
+__global__ void __launch_bounds__(256)
+tree_attn_combine_kernel(const float *__restrict__ part, bf16 *__restrict__ out, bf16 *__restrict__ out_lo,
+                         int R, int n_heads, int chunks) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int pair = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (pair >= R * n_heads) return;
+  const float *p = part + (size_t)pair * chunks * PSTRIDE;
+  float m = -INFINITY;
+  for (int c = 0; c < chunks; ++c) m = fmaxf(m, p[(size_t)c * PSTRIDE + DH]);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float l = 0.f;
+  if (m != -INFINITY) {
+    for (int c = 0; c < chunks; ++c) {
+      const float mc = p[(size_t)c * PSTRIDE + DH];
+      if (mc == -INFINITY) continue;
+      const float w = exp2f(mc - m);
+      l += w * p[(size_t)c * PSTRIDE + DH + 1];
+      const float2 a = *reinterpret_cast<const float2 *>(p + (size_t)c * PSTRIDE + 4 * lane);
+      const float2 bq = *reinterpret_cast<const float2 *>(p + (size_t)c * PSTRIDE + 4 * lane + 2);
+      acc.x += w * a.x; acc.y += w * a.y; acc.z += w * bq.x; acc.w += w * bq.y;
+    }
+  }
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+  const float v[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
+  const size_t o = (size_t)pair * DH + 4 * lane;      // pair = r * n_heads + h  ->  r * H + h * DH
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const bf16 hi = __float2bfloat16_rn(v[e]);
+    out[o + e] = hi;
+    if (out_lo != nullptr) out_lo[o + e] = __float2bfloat16_rn(v[e] - __bfloat162float(hi));
+  }
+}
+
+}  // namespace
+
+int attn_mma_chunks(int B, int n_heads, int num_sms) {
+  int c = (2 * num_sms + B * n_heads - 1) / (B * n_heads);
+  return c < 1 ? 1 : (c > 16 ? 16 : c);
+}
+
+size_t attn_mma_scratch_floats(int rows_total, int n_heads, int chunks) {
+  return (size_t)rows_total * n_heads * chunks * PSTRIDE;
+}
+
+cudaError_t tree_attention_mma(Launch L, const float *q, const void *k_cache, const void *v_cache,
+                               RowPlan plan, Operand out, float *scratch, int rows_per_seq, int B,
+                               int n_heads, int S_max, int chunks) {
+  static bool configured = false;
+  const size_t smem = 4 * (size_t)TILE_BYTES;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(tree_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int cw = (rows_per_seq + 15) / 16;
+  if (cw > 8) return cudaErrorInvalidValue;
+  const int warps = cw < 4 ? 4 : cw;
+  cudaError_t e = launch_k(tree_attn_mma_kernel, dim3(chunks, n_heads, B), dim3(warps * 32), smem, L.st, L.pdl, q,
+                           (const bf16 *)k_cache, (const bf16 *)v_cache, plan, scratch, rows_per_seq, n_heads,
+                           S_max, chunks, cw);
+  if (e != cudaSuccess) return e;
+  const int R = B * rows_per_seq;
+  return launch_k(tree_attn_combine_kernel, dim3((R * n_heads + 7) / 8), dim3(256), 0, L.st, L.pdl,
+                  (const float *)scratch, (bf16 *)out.hi, (bf16 *)out.lo, R, n_heads, chunks);
+}
+
+}  // namespace koala

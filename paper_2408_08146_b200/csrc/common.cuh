@@ -122,6 +122,13 @@ cudaError_t cast_rows(Launch L, int dtype, const float *src, const int32_t *row_
                       float *dst32, int dst32_stride, int R, int H);
 cudaError_t reduce_splits(Launch L, SplitIn P, float *Y, int ldy, int R, int ncols);
 
+// attn_mma.cu : bf16 caches, head_dim 128, tensor cores, split over key chunks
+int attn_mma_chunks(int B, int n_heads, int num_sms);
+size_t attn_mma_scratch_floats(int rows_total, int n_heads, int chunks);
+cudaError_t tree_attention_mma(Launch L, const float *q, const void *k_cache, const void *v_cache,
+                               RowPlan plan, Operand out, float *scratch, int rows_per_seq, int B,
+                               int n_heads, int S_max, int chunks);
+
 // gemm_simt.cu : Y[R][sum n_out] (fp32, ld ldy) = X[R][K_in] * W^T, X and W of `dtype`
 cudaError_t gemm_simt(Launch L, int dtype, Operand X, GemmMats m, int K_in, int R, float *Y,
                       int ldy);

@@ -55,6 +55,8 @@ struct koala_ctx {
   int M, Mp, pool, draft_rows_max, esz;
   size_t pcols;           // widest GEMM output
   // workspace
+  float *attn_part;
+  int attn_chunks;
   float *x, *qbuf, *P, *verify_logits, *draft_logits, *verify_hid, *feat[2], *mx;
   Operand xn, attn_out, act, cat, lmin;
   bool pair;              // bf16 activations kept as hi + lo
@@ -165,6 +167,10 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
   c->act = operand(F);
   c->cat = operand(2 * H);
   c->lmin = operand(H);
+  c->attn_chunks = attn_mma_chunks(B, cfg.n_heads, 148);
+  c->attn_part = (cfg.dtype == KOALA_BF16 && cfg.head_dim == 128)
+                     ? w.take<float>(attn_mma_scratch_floats(Mp, cfg.n_heads, c->attn_chunks))
+                     : nullptr;
   c->verify_tgt = w.take<int32_t>(Mp);
   c->s_parent = w.take<int32_t>(N);
   c->s_level = w.take<int32_t>(N);
@@ -283,8 +289,13 @@ int run_layer(koala_ctx *c, const LayerW &w, void *kc, void *vc, int R, int rows
   CU_TRY(rope_kv_write(LN(c), g.dtype, s, row_plan(c), c->qbuf, kc, vc, R, rows_per_seq, g.n_heads,
                        g.head_dim, g.S_max));
   const int ta = time_begin(c, KOALA_CLS_ATTENTION, 0);
-  CU_TRY(tree_attention(LN(c), g.dtype, c->qbuf, kc, vc, row_plan(c), c->attn_out, R, rows_per_seq, g.B,
-                        g.n_heads, g.head_dim, g.S_max));
+  if (c->use_tc && g.head_dim == 128 && c->attn_part != nullptr && rows_per_seq <= 128) {
+    CU_TRY(tree_attention_mma(LN(c), c->qbuf, kc, vc, row_plan(c), c->attn_out, c->attn_part, rows_per_seq,
+                              g.B, g.n_heads, g.S_max, c->attn_chunks));
+  } else {
+    CU_TRY(tree_attention(LN(c), g.dtype, c->qbuf, kc, vc, row_plan(c), c->attn_out, R, rows_per_seq, g.B,
+                          g.n_heads, g.head_dim, g.S_max));
+  }
   time_end(c, ta);
   GemmMats o{{w.wo, nullptr, nullptr}, {H, 0, 0}, 1};
   K_TRY(do_gemm(c, c->attn_out, H, o, R, nullptr, 0, &s));
