@@ -160,6 +160,7 @@ def run_koala(args):
     barrier()
     s_before = eng.seq_len.clone()
     launches_before = eng.launch_count()
+    print(f"[bench] library kernels launched before the timed region: {launches_before}", file=sys.stderr)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clocks:
         barrier()
@@ -174,6 +175,11 @@ def run_koala(args):
     assert tokens == int(sched[W:W + K].sum()), "accepted lengths do not follow the forced schedule"
     assert eng.device_status() == 0, "device status word is set"
     mean_ctx = float(s_before.float().mean().item()) + tokens / (2.0 * cfg.B)
+    if args.timed_only:
+        print(json.dumps({"metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "steps": K, "warmup": W,
+                          "ms_per_step": ms / K, "gpu_launches": launches, "note": "timed-only run"}))
+        eng.close()
+        return
 
     # ---- end to end through the public calls with host buffers: per step the forced lengths come
     #      from pinned host memory and the step's tokens are read back to the host
@@ -333,6 +339,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="koala", choices=["koala", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--timed-only", action="store_true",
+                    help="only the warm-up and the timed steps (for profiler launch lists): no end-to-end, "
+                         "per-call or per-kernel passes, no CPU baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":

@@ -98,6 +98,8 @@ def load_library(rebuild: bool = False) -> C.CDLL:
     lib.koala_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int]
     lib.koala_timing_read.restype = C.c_int
     lib.koala_timing_read.argtypes = [C.c_void_p, C.POINTER(koala_timing)]
+    lib.koala_set_tuning.restype = None
+    lib.koala_set_tuning.argtypes = [C.c_int, C.c_int]
     lib.koala_launch_count.restype = C.c_uint64
     lib.koala_launch_count.argtypes = []
     lib.koala_poll.restype = C.c_int

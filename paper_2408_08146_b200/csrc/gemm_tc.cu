@@ -39,6 +39,7 @@ constexpr int W_STAGE_BYTES = BM * BK * 2;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // about a second of SM clock
 constexpr int E_TIMEOUT = 6;
 constexpr int MAX_STAGES = 12;
+constexpr int L2_AHEAD = 8;          // weight tiles (16 KB each) prefetched into L2 beyond the ring
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -195,6 +196,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
         tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, (kb_lo + it) * BK, row0);
       }
+      // and a few more of this CTA's weight tiles are requested into L2 while the producer of X
+      // runs (bounded, so that all CTAs together stay well inside the L2)
+      const int ahead = nkb < pre + L2_AHEAD ? nkb : pre + L2_AHEAD;
+      for (int it = pre; it < ahead; ++it)
+        asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+                     ::"l"(tmW), "r"((kb_lo + it) * BK), "r"(row0) : "memory");
       pdl_wait();
       const int lo_off = P.tt * BK * 2;          // the lo rows follow the hi rows of the tile
       for (int it = 0; it < pre; ++it) {
@@ -295,6 +302,8 @@ std::mutex g_mu;
 std::map<std::tuple<const void *, int, int, int>, CUtensorMap> g_maps;   // (ptr, rows, K, box rows)
 int g_smem_optin = 0;
 int g_num_sms = 148;
+int g_tune_stages = 0;      // 0 = as many as fit (at most 8)
+int g_tune_max_split = 0;   // 0 = default rule
 
 bool get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out) {
   std::lock_guard<std::mutex> lock(g_mu);
@@ -344,6 +353,11 @@ int tc_init_driver(char *err, size_t errlen) {
   return 0;
 }
 
+void tc_set_tuning(int key, int value) {
+  if (key == 1) g_tune_stages = value;
+  if (key == 2) g_tune_max_split = value;
+}
+
 void tc_forget_maps() {
   std::lock_guard<std::mutex> lock(g_mu);
   g_maps.clear();
@@ -361,7 +375,8 @@ bool tc_supported(const GemmMats &m, int K_in) {
 int tc_default_split(int n_tiles, int kblocks) {
   int best = 1;
   double best_eff = 0.0;
-  const int max_split = kblocks / 8 > 0 ? (kblocks / 8 < 16 ? kblocks / 8 : 16) : 1;
+  int max_split = kblocks / 8 > 0 ? (kblocks / 8 < 16 ? kblocks / 8 : 16) : 1;
+  if (g_tune_max_split > 0 && max_split > g_tune_max_split) max_split = g_tune_max_split;
   for (int s = 1; s <= max_split; ++s) {
     const int ctas = n_tiles * s;
     const int waves = (ctas + g_num_sms - 1) / g_num_sms;
@@ -417,6 +432,11 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   int stages = (g_smem_optin - 2048) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages > 8) stages = 8;
+  // default: two CTAs per SM (each with half of the shared memory), so that one CTA's prologue and
+  // epilogue overlap the other's streaming
+  const int two_per_sm = (g_smem_optin / 2 - 2048) / stage_bytes;
+  if (g_tune_stages == 0 && two_per_sm >= 2 && two_per_sm < stages) stages = two_per_sm;
+  if (g_tune_stages > 0 && g_tune_stages < stages) stages = g_tune_stages;
   if (stages < 2) return cudaErrorInvalidValue;
   P.stages = stages;
   CUtensorMap mw[3], mx, mxlo;

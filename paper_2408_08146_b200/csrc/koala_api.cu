@@ -13,6 +13,7 @@ using namespace koala;
 
 namespace koala {
 void tc_forget_maps();
+void tc_set_tuning(int key, int value);
 unsigned long long g_launches = 0;
 }
 
@@ -644,6 +645,8 @@ int koala_timing_read(koala_ctx *c, koala_timing *out) {
   (void)cudaGetLastError();
   return KOALA_OK;
 }
+
+void koala_set_tuning(int key, int value) { koala::tc_set_tuning(key, value); }
 
 uint64_t koala_launch_count(void) { return (uint64_t)koala::g_launches; }
 

@@ -89,6 +89,99 @@ __global__ void row_epilogue_kernel(int mode, float *__restrict__ x, SplitIn P,
   }
 }
 
+// Vectorised variant for H % 4 == 0: one CTA per row, every thread owns up to VPT groups of four
+// consecutive columns, keeps them in registers between the two passes and issues all split-K
+// partial loads of a group back to back.
+__device__ __forceinline__ float4 split_sum4(const SplitIn &P, int r, int c) {
+  const float *q = P.p + (size_t)r * P.ld + c;
+  float4 v = *reinterpret_cast<const float4 *>(q);
+  for (int s = 1; s < P.n; ++s) {
+    const float4 u = *reinterpret_cast<const float4 *>(q + (size_t)s * P.stride);
+    v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
+  }
+  return v;
+}
+template <typename T> __device__ __forceinline__ float4 load4(const T *p);
+template <> __device__ __forceinline__ float4 load4<float>(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+template <> __device__ __forceinline__ float4 load4<bf16>(const bf16 *p) {
+  const uint2 u = *reinterpret_cast<const uint2 *>(p);
+  const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u.x));
+  const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u.y));
+  return make_float4(a.x, a.y, b.x, b.y);
+}
+__device__ __forceinline__ void store_operand4(float *hi, float *lo, size_t i, float4 v) {
+  (void)lo;
+  *reinterpret_cast<float4 *>(hi + i) = v;
+}
+__device__ __forceinline__ void store_operand4(bf16 *hi, bf16 *lo, size_t i, float4 v) {
+  const __nv_bfloat162 h0 = __floats2bfloat162_rn(v.x, v.y), h1 = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<const uint32_t *>(&h0);
+  u.y = *reinterpret_cast<const uint32_t *>(&h1);
+  *reinterpret_cast<uint2 *>(hi + i) = u;
+  if (lo != nullptr) {
+    const float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
+    const __nv_bfloat162 l0 = __floats2bfloat162_rn(v.x - f0.x, v.y - f0.y);
+    const __nv_bfloat162 l1 = __floats2bfloat162_rn(v.z - f1.x, v.w - f1.y);
+    u.x = *reinterpret_cast<const uint32_t *>(&l0);
+    u.y = *reinterpret_cast<const uint32_t *>(&l1);
+    *reinterpret_cast<uint2 *>(lo + i) = u;
+  }
+}
+
+template <typename T, int VPT>
+__global__ void __launch_bounds__(1024)
+row_epilogue_vec_kernel(int mode, float *__restrict__ x, SplitIn P, const T *__restrict__ bias,
+                        const T *__restrict__ g, T *__restrict__ xn, T *__restrict__ xn_lo,
+                        float *__restrict__ out_f32, int H, float eps) {
+  __shared__ float red[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  float *xr = x + (size_t)r * H;
+  float4 v[VPT];
+  float ss = 0.f;
+#pragma unroll
+  for (int k = 0; k < VPT; ++k) {
+    const int c = (threadIdx.x + k * blockDim.x) * 4;
+    if (c < H) {
+      const float4 p = split_sum4(P, r, c);
+      float4 o;
+      if (mode == 0) {
+        const float4 xv = *reinterpret_cast<const float4 *>(xr + c);
+        o = make_float4(xv.x + p.x, xv.y + p.y, xv.z + p.z, xv.w + p.w);
+      } else {
+        const float4 b = load4<T>(bias + c);
+        if (mode == 1) {
+          o = make_float4(p.x + b.x, p.y + b.y, p.z + b.z, p.w + b.w);
+        } else {
+          const float4 xv = *reinterpret_cast<const float4 *>(xr + c);
+          o = make_float4(xv.x + silu_f(p.x + b.x), xv.y + silu_f(p.y + b.y), xv.z + silu_f(p.z + b.z),
+                          xv.w + silu_f(p.w + b.w));
+        }
+      }
+      *reinterpret_cast<float4 *>(xr + c) = o;
+      v[k] = o;
+      ss += o.x * o.x + o.y * o.y + o.z * o.z + o.w * o.w;
+    }
+  }
+  float inv = 1.f;
+  if (g != nullptr) inv = rsqrtf(block_sum(ss, red) / (float)H + eps);
+#pragma unroll
+  for (int k = 0; k < VPT; ++k) {
+    const int c = (threadIdx.x + k * blockDim.x) * 4;
+    if (c < H) {
+      float4 n = v[k];
+      if (g != nullptr) {
+        const float4 gg = load4<T>(g + c);
+        n = make_float4(n.x * inv * gg.x, n.y * inv * gg.y, n.z * inv * gg.z, n.w * inv * gg.w);
+      }
+      if (xn != nullptr) store_operand4(xn, xn_lo, (size_t)r * H + c, n);
+      if (out_f32 != nullptr) *reinterpret_cast<float4 *>(out_f32 + (size_t)r * H + c) = n;
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------- EAGLE fc input
 template <typename T>
 __global__ void eagle_concat_kernel(const float *__restrict__ feat_src,
@@ -161,6 +254,50 @@ __global__ void rope_kv_kernel(SplitIn qkv, RowPlan plan, float *__restrict__ q_
   v_cache[base + i + half] = from_f<T>(v1);
 }
 
+// One CTA per row; a thread rotates two adjacent pairs (i, i+1) and (i + half, i + half + 1) of
+// one head with 8-byte loads.
+__device__ __forceinline__ float2 split_sum2(const SplitIn &P, int r, int c) {
+  const float *q = P.p + (size_t)r * P.ld + c;
+  float2 v = *reinterpret_cast<const float2 *>(q);
+  for (int s = 1; s < P.n; ++s) {
+    const float2 u = *reinterpret_cast<const float2 *>(q + (size_t)s * P.stride);
+    v.x += u.x; v.y += u.y;
+  }
+  return v;
+}
+__device__ __forceinline__ void store2(float *p, float a, float b) { *reinterpret_cast<float2 *>(p) = make_float2(a, b); }
+__device__ __forceinline__ void store2(bf16 *p, float a, float b) {
+  *reinterpret_cast<__nv_bfloat162 *>(p) = __floats2bfloat162_rn(a, b);
+}
+template <typename T>
+__global__ void __launch_bounds__(1024)
+rope_kv_vec_kernel(SplitIn qkv, RowPlan plan, float *__restrict__ q_out, T *__restrict__ k_cache,
+                   T *__restrict__ v_cache, int rows_per_seq, int n_heads, int head_dim, int S_max) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  const int half = head_dim >> 1, H = n_heads * head_dim, hq = half >> 1;
+  const int b = r / rows_per_seq;
+  const int slot = plan.slot[r];
+  const bool wr = slot >= 0 && slot < S_max;
+  for (int p = threadIdx.x; p < n_heads * hq; p += blockDim.x) {
+    const int h = p / hq, i = (p - h * hq) * 2;
+    const float4 cs = *reinterpret_cast<const float4 *>(&plan.rope[(size_t)r * half + i]);   // c0 s0 c1 s1
+    const int c0 = h * head_dim + i, c1 = c0 + half;
+    const float2 qa = split_sum2(qkv, r, c0), qb = split_sum2(qkv, r, c1);
+    store2(q_out + (size_t)r * H + c0, qa.x * cs.x - qb.x * cs.y, qa.y * cs.z - qb.y * cs.w);
+    store2(q_out + (size_t)r * H + c1, qb.x * cs.x + qa.x * cs.y, qb.y * cs.z + qa.y * cs.w);
+    if (!wr) continue;
+    const float2 ka = split_sum2(qkv, r, H + c0), kb = split_sum2(qkv, r, H + c1);
+    const float2 va = split_sum2(qkv, r, 2 * H + c0), vb = split_sum2(qkv, r, 2 * H + c1);
+    const size_t base = (((size_t)b * n_heads + h) * S_max + slot) * head_dim + i;
+    store2(k_cache + base, ka.x * cs.x - kb.x * cs.y, ka.y * cs.z - kb.y * cs.w);
+    store2(k_cache + base + half, kb.x * cs.x + ka.x * cs.y, kb.y * cs.z + ka.y * cs.w);
+    store2(v_cache + base, va.x, va.y);
+    store2(v_cache + base + half, vb.x, vb.y);
+  }
+}
+
 // ------------------------------------------------------------------------------- SwiGLU
 template <typename T>
 __global__ void swiglu_kernel(SplitIn gu, T *__restrict__ act, T *__restrict__ act_lo, int F) {
@@ -170,6 +307,18 @@ __global__ void swiglu_kernel(SplitIn gu, T *__restrict__ act, T *__restrict__ a
   const int f = blockIdx.x * blockDim.x + threadIdx.x;
   if (f >= F) return;
   store_operand(act, act_lo, (size_t)r * F + f, silu_f(gu.at(r, f)) * gu.at(r, F + f));
+}
+
+template <typename T>
+__global__ void swiglu_vec_kernel(SplitIn gu, T *__restrict__ act, T *__restrict__ act_lo, int F) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.y;
+  const int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (f >= F) return;
+  const float4 a = split_sum4(gu, r, f), b = split_sum4(gu, r, F + f);
+  store_operand4(act, act_lo, (size_t)r * F + f,
+                 make_float4(silu_f(a.x) * b.x, silu_f(a.y) * b.y, silu_f(a.z) * b.z, silu_f(a.w) * b.w));
 }
 
 // ------------------------------------------------------------------------------- tree attention
@@ -345,6 +494,19 @@ cudaError_t embed_norm(Launch L, int dtype, const int32_t *tok, const void *E, c
 
 cudaError_t row_epilogue(Launch L, int dtype, int mode, float *x, SplitIn P, const void *bias,
                          const void *g, Operand xn, float *out_f32, int R, int H, float eps) {
+  if (H % 4 == 0 && P.ld % 4 == 0 && P.stride % 4 == 0 && H <= 8192) {
+    const int groups = H / 4;
+    int threads = groups <= 1024 ? ((groups + 31) / 32) * 32 : (((groups + 1) / 2 + 31) / 32) * 32;
+    if (groups <= 1024) {
+      DISPATCH_T(dtype, return launch_k(row_epilogue_vec_kernel<T, 1>, dim3(R), dim3(threads), 0, L.st, L.pdl,
+                                        mode, x, P, (const T *)bias, (const T *)g, (T *)xn.hi, (T *)xn.lo,
+                                        out_f32, H, eps);)
+    } else {
+      DISPATCH_T(dtype, return launch_k(row_epilogue_vec_kernel<T, 2>, dim3(R), dim3(threads), 0, L.st, L.pdl,
+                                        mode, x, P, (const T *)bias, (const T *)g, (T *)xn.hi, (T *)xn.lo,
+                                        out_f32, H, eps);)
+    }
+  }
   DISPATCH_T(dtype, return launch_k(row_epilogue_kernel<T>, dim3(R), dim3(256), 0, L.st, L.pdl, mode,
                                     x, P, (const T *)bias, (const T *)g, (T *)xn.hi, (T *)xn.lo, out_f32,
                                     H, eps);)
@@ -371,12 +533,23 @@ cudaError_t reduce_splits(Launch L, SplitIn P, float *Y, int ldy, int R, int nco
 cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowPlan plan, float *q_out,
                           void *k_cache, void *v_cache, int R, int rows_per_seq, int n_heads,
                           int head_dim, int S_max) {
+  if (head_dim % 4 == 0 && qkv.ld % 2 == 0 && qkv.stride % 2 == 0) {
+    const int work = n_heads * head_dim / 4;
+    const int threads = work < 1024 ? ((work + 31) / 32) * 32 : 1024;
+    DISPATCH_T(dtype, return launch_k(rope_kv_vec_kernel<T>, dim3(R), dim3(threads), 0, L.st, L.pdl, qkv, plan,
+                                      q_out, (T *)k_cache, (T *)v_cache, rows_per_seq, n_heads, head_dim,
+                                      S_max);)
+  }
   DISPATCH_T(dtype, return launch_k(rope_kv_kernel<T>, dim3(R, n_heads), dim3(head_dim / 2), 0, L.st,
                                     L.pdl, qkv, plan, q_out, (T *)k_cache, (T *)v_cache,
                                     rows_per_seq, n_heads, head_dim, S_max);)
 }
 
 cudaError_t swiglu(Launch L, int dtype, SplitIn gu, Operand act, int R, int F) {
+  if (F % 4 == 0 && gu.ld % 4 == 0 && gu.stride % 4 == 0) {
+    DISPATCH_T(dtype, return launch_k(swiglu_vec_kernel<T>, dim3((F / 4 + 255) / 256, R), dim3(256), 0, L.st,
+                                      L.pdl, gu, (T *)act.hi, (T *)act.lo, F);)
+  }
   DISPATCH_T(dtype, return launch_k(swiglu_kernel<T>, dim3((F + 255) / 256, R), dim3(256), 0, L.st,
                                     L.pdl, gu, (T *)act.hi, (T *)act.lo, F);)
 }
