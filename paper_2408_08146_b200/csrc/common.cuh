@@ -136,7 +136,7 @@ cudaError_t gemm_simt(Launch L, int dtype, Operand X, GemmMats m, int K_in, int 
 // gemm_tc.cu : bf16 tensor-core path; writes `split` partial matrices `split_stride` apart.
 int tc_init_driver(char *err, size_t errlen);   // 0 on success
 bool tc_supported(const GemmMats &m, int K_in);
-int tc_default_split(int n_tiles, int kblocks);
+int tc_default_split(int n_tiles, int kblocks, int tokens);
 cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in, int R,
                     float *Y, int ldy, int split, size_t split_stride, int *status);
 

@@ -370,23 +370,18 @@ bool tc_supported(const GemmMats &m, int K_in) {
   return g_encode != nullptr;
 }
 
-// Split so that tiles x split comes close to a whole number of waves of the SMs, while every
-// split keeps at least 8 K-blocks.
-int tc_default_split(int n_tiles, int kblocks) {
-  int best = 1;
-  double best_eff = 0.0;
-  int max_split = kblocks / 8 > 0 ? (kblocks / 8 < 16 ? kblocks / 8 : 16) : 1;
-  if (g_tune_max_split > 0 && max_split > g_tune_max_split) max_split = g_tune_max_split;
-  for (int s = 1; s <= max_split; ++s) {
-    const int ctas = n_tiles * s;
-    const int waves = (ctas + g_num_sms - 1) / g_num_sms;
-    const double eff = (double)ctas / ((double)waves * g_num_sms);
-    if (eff > best_eff + 0.03) {
-      best_eff = eff;
-      best = s;
-    }
-  }
-  return best;
+// Split-K factor: as many CTAs as fit in one wave of the co-resident slots (two per SM), while
+// every split keeps at least 8 K-blocks and the fp32 partial sums written and re-read
+// (split x tokens x 4 bytes per output) stay below about half of the weight bytes.
+int tc_default_split(int n_tiles, int kblocks, int tokens) {
+  const int slots = 2 * g_num_sms;
+  int s = slots / (n_tiles > 0 ? n_tiles : 1);
+  const int by_k = kblocks / 8;
+  const int by_traffic = (kblocks * 64) / (8 * (tokens > 0 ? tokens : 1));
+  if (s > by_k) s = by_k;
+  if (s > by_traffic) s = by_traffic;
+  if (g_tune_max_split > 0 && s > g_tune_max_split) s = g_tune_max_split;
+  return s < 1 ? 1 : s;
 }
 
 cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in, int R,

@@ -255,7 +255,7 @@ int do_gemm(koala_ctx *c, Operand X, int K_in, GemmMats m, int R, float *direct,
   if (c->use_tc && c->cfg.dtype == KOALA_BF16 && tc_supported(m, K_in)) {
     int tiles = 0;
     for (int i = 0; i < m.n; ++i) tiles += (m.n_out[i] + 127) / 128;
-    int split = direct ? 1 : tc_default_split(tiles, K_in / 64);
+    int split = direct ? 1 : tc_default_split(tiles, K_in / 64, R);
     if (split > MAX_SPLIT) split = MAX_SPLIT;
     const size_t stride = (size_t)c->Mp * ld;
     const int tb = time_begin(c, KOALA_CLS_GEMM_TC, wbytes);
@@ -707,7 +707,7 @@ int koala_gemm_bf16(const void *X, const void *X_lo, const void *W, float *Y, in
   char e[160];
   if (tc_init_driver(e, sizeof(e)) != 0) return KOALA_E_CUDA;
   if (!tc_supported(m, K_in)) return KOALA_E_UNSUPPORTED;
-  int split = split_k > 0 ? split_k : tc_default_split((N_out + 127) / 128, K_in / 64);
+  int split = split_k > 0 ? split_k : tc_default_split((N_out + 127) / 128, K_in / 64, M);
   if (split > MAX_SPLIT) split = MAX_SPLIT;
   if (split > K_in / 64) split = K_in / 64;
   // X must hold a whole token tile: the caller's buffer has M rows, rounded up by the map's
