@@ -121,6 +121,16 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def reduce_over_ranks(times_ms, counts, dist=None, device="cpu"):
+    """Whole-job figures from per-rank ones: MAX of the times, SUM of the counts (replicas)."""
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    n = torch.tensor(list(counts), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return [float(v) for v in t], [float(v) for v in n]
+
+
 # ------------------------------------------------------------------------------------------------
 def run_koala(args):
     from paper_2408_08146_b200 import Koala
@@ -224,12 +234,8 @@ def run_koala(args):
     ab = algorithmic_bytes_per_step(cfg, mean_ctx)
 
     # ---- reduce over ranks
-    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
-    n = torch.tensor([tokens, tokens_e2e, launches], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(n, op=dist.ReduceOp.SUM)
-    ms_max, ms_e2e_max = float(t[0]), float(t[1])
+    t, n = reduce_over_ranks([ms, ms_e2e], [tokens, tokens_e2e, launches], dist, dev)
+    ms_max, ms_e2e_max = t[0], t[1]
     line = {
         "metric": METRIC, "value": float(n[0]) / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak",

@@ -77,7 +77,7 @@ def load_library(rebuild: bool = False) -> C.CDLL:
     global _lib
     if _lib is not None and not rebuild:
         return _lib
-    path = _build.build(force=rebuild)
+    path = os.environ.get("KOALA_LIBRARY") or _build.build(force=rebuild)   # an explicit library wins
     lib = C.CDLL(path)
     lib.koala_workspace_bytes.restype = C.c_size_t
     lib.koala_workspace_bytes.argtypes = [C.POINTER(koala_config)]

@@ -23,7 +23,10 @@ def assert_close(gpu, ref, dtype, what, atol=None, rtol=None):
     bad = ~((err <= atol) | (err <= rtol * np.abs(ref)))
     assert not bad.any(), (f"{what}: {bad.sum()} of {bad.size} elements out of tolerance; "
                            f"max abs err {err.max():.3e} (ref scale {np.abs(ref).max():.3e})")
-    return float(err.max())
+    if err.size:
+        print(f"[parity] {what}: max abs err {err.max():.3e}, rms err {np.sqrt(np.mean(err ** 2)):.3e}, "
+              f"ref rms {np.sqrt(np.mean(ref ** 2)):.3e}")
+    return float(err.max()) if err.size else 0.0
 
 
 def check_argmax(gpu_idx, ref_logits, what):
