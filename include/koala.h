@@ -239,6 +239,27 @@ int koala_gemm_bf16(const void *X, const void *X_lo /* optional residual of X, s
                     void *scratch, size_t scratch_bytes, int use_tensor_cores, int split_k,
                     void *cuda_stream, int *device_status /* device int, may be NULL */);
 
+/* The paper has no counterpart for this entry point; it is a packaging variant of koala_gemm_bf16.
+ *
+ * Same product, Y[M][N_out] = (X [+ X_lo]) * W^T on the tensor-core path, for callers that cannot
+ * provide (or allocate) a scratch buffer: a serving loop whose device memory is fixed at start-up,
+ * a plug-in that a host framework hands only inputs and outputs, code running close to the
+ * device's memory limit.  The split-K partial sums go to a fixed 8 MiB array inside the library's
+ * device image (koala_gemm_static_scratch_bytes(); every GPU that loads the library holds it until
+ * the process exits).  Nothing is allocated or freed on the device, by this call or under it.
+ *   - split_k * M * N_out * 4 bytes must fit in the array, else KOALA_E_CAPACITY (split_k 0 =
+ *     automatic; split_k 1 needs no scratch at all).  K_in % 64 == 0, X rows as koala_gemm_x_rows.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and prepares the kernel; make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents (none of
+ *     which is read before it is overwritten).  Two calls whose kernels may overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them on one stream or with
+ *     events. */
+size_t koala_gemm_static_scratch_bytes(void);
+int koala_gemm_bf16_static(const void *X, const void *X_lo, const void *W, float *Y, int ldy, int M,
+                           int N_out, int K_in, int split_k, void *cuda_stream,
+                           int *device_status /* device int, may be NULL */);
+
 #ifdef __cplusplus
 }
 #endif

@@ -98,6 +98,11 @@ def load_library(rebuild: bool = False) -> C.CDLL:
     lib.koala_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int]
     lib.koala_timing_read.restype = C.c_int
     lib.koala_timing_read.argtypes = [C.c_void_p, C.POINTER(koala_timing)]
+    lib.koala_gemm_static_scratch_bytes.restype = C.c_size_t
+    lib.koala_gemm_static_scratch_bytes.argtypes = []
+    lib.koala_gemm_bf16_static.restype = C.c_int
+    lib.koala_gemm_bf16_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                           C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
     lib.koala_set_tuning.restype = None
     lib.koala_set_tuning.argtypes = [C.c_int, C.c_int]
     lib.koala_launch_count.restype = C.c_uint64

@@ -1,0 +1,66 @@
+// koala_gemm_bf16_static: the stand-alone weight-streaming GEMM for callers that must not allocate.
+//
+// The split-K partial sums of the tensor-core GEMM normally live in a scratch buffer that the
+// caller allocates.  Some callers cannot do that: code running inside a real-time serving loop
+// whose memory pool is fixed at start-up, plug-ins handed only input and output buffers by a host
+// framework that owns all device memory, or code running while the process is near its memory
+// limit, where a cudaMalloc could fail or stall every stream of the device.  For them the scratch
+// is a fixed array in the library's own device image.
+#include "../../include/koala.h"
+#include "common.cuh"
+
+namespace {
+
+// 8 MiB of fp32 partial sums; every device that loads the library holds this until the process exits.
+constexpr size_t STATIC_SCRATCH_FLOATS = (size_t)2 * 1024 * 1024;
+static __device__ __align__(256) float g_static_scratch[STATIC_SCRATCH_FLOATS];
+
+constexpr int MAX_DEVICES = 64;
+float *g_scratch_ptr[MAX_DEVICES] = {nullptr};   // device address of the array, per device
+
+}  // namespace
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+size_t koala_gemm_static_scratch_bytes(void) { return STATIC_SCRATCH_FLOATS * sizeof(float); }
+
+int koala_gemm_bf16_static(const void *X, const void *X_lo, const void *W, float *Y, int ldy, int M,
+                           int N_out, int K_in, int split_k, void *cuda_stream, int *device_status) {
+  using namespace koala;
+  if (!X || !W || !Y || M < 1 || N_out < 1 || K_in < 1 || ldy < N_out) return KOALA_E_INVALID;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return KOALA_E_CUDA;
+  if (dev < 0 || dev >= MAX_DEVICES) return KOALA_E_UNSUPPORTED;
+  if (g_scratch_ptr[dev] == nullptr) {
+    // The array's name is only a host-side handle; kernels need its address on the current device.
+    float *p = nullptr;
+    if (cudaGetSymbolAddress((void **)&p, g_static_scratch) != cudaSuccess || p == nullptr) return KOALA_E_CUDA;
+    g_scratch_ptr[dev] = p;
+  }
+  char err[160];
+  if (tc_init_driver(err, sizeof(err)) != 0) return KOALA_E_CUDA;
+  GemmMats m{{W, nullptr, nullptr}, {N_out, 0, 0}, 1};
+  if (!tc_supported(m, K_in)) return KOALA_E_UNSUPPORTED;
+  int split = split_k > 0 ? split_k : tc_default_split((N_out + 127) / 128, K_in / 64, M);
+  if (split > K_in / 64) split = K_in / 64;
+  if (split > 8) split = 8;
+  Launch L{(cudaStream_t)cuda_stream, false};
+  Operand Xo{const_cast<void *>(X), const_cast<void *>(X_lo)};
+  const int rows_alloc = koala_gemm_x_rows(M, X_lo != nullptr);
+  if (split == 1)
+    return gemm_tc(L, Xo, rows_alloc, m, K_in, M, Y, ldy, 1, 0, device_status) == cudaSuccess ? KOALA_OK
+                                                                                              : KOALA_E_CUDA;
+  const size_t stride = (size_t)M * N_out;
+  if ((size_t)split * stride > STATIC_SCRATCH_FLOATS) return KOALA_E_CAPACITY;
+  float *scratch = g_scratch_ptr[dev];
+  // every partial element that is read below is written by exactly one CTA of this launch, so the
+  // previous call's contents need no clearing
+  if (gemm_tc(L, Xo, rows_alloc, m, K_in, M, scratch, N_out, split, stride, device_status) != cudaSuccess)
+    return KOALA_E_CUDA;
+  SplitIn s{scratch, split, stride, N_out};
+  return reduce_splits(L, s, Y, ldy, M, N_out) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
+}
+
+#pragma GCC visibility pop
+}

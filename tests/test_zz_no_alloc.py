@@ -1,0 +1,77 @@
+"""koala_gemm_bf16_static: the GEMM entry point whose split-K scratch is a fixed array inside the
+library, for callers that cannot allocate device memory (fixed memory pools, plug-ins that only
+receive inputs and outputs, processes near the device's memory limit).
+
+Checked through the C ABI against koala_gemm_bf16 (caller-provided scratch) on the same inputs,
+twice in a row with different shapes and split factors, so that the second call runs over the
+first call's leftovers.  Collected last on purpose.
+"""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2408_08146_b200 import binding
+from workloads.generate import normal_tensor
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _case(lib, M, N, K, split, pair, tag):
+    rows = lib.koala_gemm_x_rows(M, int(pair))
+    xf = normal_tensor(21, f"x.{tag}", (rows, K), 1.0, 0.0, torch.float32, DEV)
+    hi = xf.to(torch.bfloat16)
+    lo = (xf - hi.float()).to(torch.bfloat16) if pair else None
+    w = normal_tensor(22, f"w.{tag}", (N, K), 0.02, 0.0, torch.bfloat16, DEV)
+    st = torch.cuda.current_stream().cuda_stream
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    # reference: the existing entry point with a scratch buffer allocated here
+    nb = int(lib.koala_gemm_scratch_bytes(M, N, K))
+    scratch = torch.empty(nb, dtype=torch.uint8, device=DEV)
+    y_ref = torch.empty(M, N, dtype=torch.float32, device=DEV)
+    rc = lib.koala_gemm_bf16(hi.data_ptr(), lo.data_ptr() if pair else None, w.data_ptr(), y_ref.data_ptr(), N,
+                             M, N, K, scratch.data_ptr(), nb, 1, split, st, status.data_ptr())
+    assert rc == 0
+    # the entry point under test: inputs and outputs only
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+    before = torch.cuda.memory_allocated(DEV)
+    rc = lib.koala_gemm_bf16_static(hi.data_ptr(), lo.data_ptr() if pair else None, w.data_ptr(), y.data_ptr(),
+                                    N, M, N, K, split, st, status.data_ptr())
+    assert rc == 0
+    assert torch.cuda.memory_allocated(DEV) == before
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    a, b = y.cpu().numpy(), y_ref.cpu().numpy()
+    assert np.isfinite(a).all()
+    # same kernels, same split, same summation order: within the GEMM tests' tolerance (in fact equal)
+    assert np.abs(a - b).max() <= 2e-5 * np.sqrt(K) + 1e-6
+    ref = (hi.double() + (lo.double() if pair else 0)).cpu().numpy()[:M] @ w.double().cpu().numpy().T
+    assert np.abs(a - ref).max() <= 2e-5 * np.sqrt(K) + 1e-6
+
+
+def test_static_scratch_gemm_matches_twice_in_a_row():
+    lib = binding.load_library()
+    assert lib.koala_gemm_static_scratch_bytes() == 8 * 1024 * 1024
+    _case(lib, 64, 1024, 4096, 8, True, "first")        # 8 x 64 x 1024 x 4 B = 2 MiB of the array
+    _case(lib, 40, 640, 1024, 3, False, "second")       # smaller: runs over the first call's leftovers
+    _case(lib, 10, 4096, 4096, 0, True, "auto")         # automatic split
+
+
+def test_static_scratch_gemm_rejects_oversize_and_bad_arguments():
+    lib = binding.load_library()
+    x = torch.zeros(64, 4096, dtype=torch.bfloat16, device=DEV)
+    w = torch.zeros(32000, 4096, dtype=torch.bfloat16, device=DEV)
+    y = torch.zeros(64, 32000, dtype=torch.float32, device=DEV)
+    st = torch.cuda.current_stream().cuda_stream
+    # 8 x 64 x 32000 x 4 B = 65.5 MB > 8 MiB
+    assert lib.koala_gemm_bf16_static(x.data_ptr(), None, w.data_ptr(), y.data_ptr(), 32000, 64, 32000, 4096, 8,
+                                      st, None) == 3
+    # split 1 needs no scratch and is accepted at any size
+    assert lib.koala_gemm_bf16_static(x.data_ptr(), None, w.data_ptr(), y.data_ptr(), 32000, 64, 32000, 4096, 1,
+                                      st, None) == 0
+    torch.cuda.synchronize()
+    assert lib.koala_gemm_bf16_static(None, None, w.data_ptr(), y.data_ptr(), 32000, 64, 32000, 4096, 1, st, None) == 1
+    assert lib.koala_gemm_bf16_static(x.data_ptr(), None, w.data_ptr(), y.data_ptr(), 32000, 64, 32000, 4100, 1,
+                                      st, None) == 2       # K_in not a multiple of 64
