@@ -123,7 +123,7 @@ cudaError_t cast_rows(Launch L, int dtype, const float *src, const int32_t *row_
 cudaError_t reduce_splits(Launch L, SplitIn P, float *Y, int ldy, int R, int ncols);
 
 // attn_mma.cu : bf16 caches, head_dim 128, tensor cores, split over key chunks
-int attn_mma_chunks(int B, int n_heads, int num_sms);
+int attn_mma_chunks(int B, int n_heads, int rows_per_seq, int S_max, int num_sms);
 size_t attn_mma_scratch_floats(int rows_total, int n_heads, int chunks);
 cudaError_t tree_attention_mma(Launch L, const float *q, const void *k_cache, const void *v_cache,
                                RowPlan plan, Operand out, float *scratch, int rows_per_seq, int B,

@@ -168,7 +168,7 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
   c->act = operand(F);
   c->cat = operand(2 * H);
   c->lmin = operand(H);
-  c->attn_chunks = attn_mma_chunks(B, cfg.n_heads, 148);
+  c->attn_chunks = 16;     // largest chunk count any launch may choose
   c->attn_part = (cfg.dtype == KOALA_BF16 && cfg.head_dim == 128)
                      ? w.take<float>(attn_mma_scratch_floats(Mp, cfg.n_heads, c->attn_chunks))
                      : nullptr;
@@ -292,7 +292,8 @@ int run_layer(koala_ctx *c, const LayerW &w, void *kc, void *vc, int R, int rows
   const int ta = time_begin(c, KOALA_CLS_ATTENTION, 0);
   if (c->use_tc && g.head_dim == 128 && c->attn_part != nullptr && rows_per_seq <= 128) {
     CU_TRY(tree_attention_mma(LN(c), c->qbuf, kc, vc, row_plan(c), c->attn_out, c->attn_part, rows_per_seq,
-                              g.B, g.n_heads, g.S_max, c->attn_chunks));
+                              g.B, g.n_heads, g.S_max,
+                              attn_mma_chunks(g.B, g.n_heads, rows_per_seq, g.S_max, 148)));
   } else {
     CU_TRY(tree_attention(LN(c), g.dtype, c->qbuf, kc, vc, row_plan(c), c->attn_out, R, rows_per_seq, g.B,
                           g.n_heads, g.head_dim, g.S_max));
