@@ -113,9 +113,22 @@ tree_attn_mma_kernel(const float *__restrict__ q, const bf16 *__restrict__ kc, c
   const int i0 = rg * 16 + g, i1 = i0 + 8;
   const bool in0 = i0 < rows_per_seq, in1 = i1 < rows_per_seq;
   const int r0 = b * rows_per_seq + (in0 ? i0 : 0), r1 = b * rows_per_seq + (in1 ? i1 : 0);
-  const bool ok0 = in0 && plan.slot[r0] >= 0, ok1 = in1 && plan.slot[r1] >= 0;
-  const uint64_t m00 = ok0 ? plan.mask[(size_t)r0 * 2] : 0ull, m01 = ok0 ? plan.mask[(size_t)r0 * 2 + 1] : 0ull;
-  const uint64_t m10 = ok1 ? plan.mask[(size_t)r1 * 2] : 0ull, m11 = ok1 ? plan.mask[(size_t)r1 * 2 + 1] : 0ull;
+  // every global load of the prologue is issued before the first use of any of them
+  const int slot0 = plan.slot[r0], slot1 = plan.slot[r1];
+  const uint64_t mk00 = plan.mask[(size_t)r0 * 2], mk01 = plan.mask[(size_t)r0 * 2 + 1];
+  const uint64_t mk10 = plan.mask[(size_t)r1 * 2], mk11 = plan.mask[(size_t)r1 * 2 + 1];
+  float2 qa[8][4];
+  {
+    const float *q0 = q + (size_t)r0 * H + h * DH, *q1 = q + (size_t)r1 * H + h * DH;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      const int col = ks * 16 + 2 * t;
+      qa[ks][0] = *reinterpret_cast<const float2 *>(q0 + col);
+      qa[ks][1] = *reinterpret_cast<const float2 *>(q1 + col);
+      qa[ks][2] = *reinterpret_cast<const float2 *>(q0 + col + 8);
+      qa[ks][3] = *reinterpret_cast<const float2 *>(q1 + col + 8);
+    }
+  }
 
 #pragma unroll
   for (int sidx = 0; sidx < NST - 1; ++sidx) {
@@ -123,21 +136,17 @@ tree_attn_mma_kernel(const float *__restrict__ q, const bf16 *__restrict__ kc, c
     cp_async_commit();
   }
 
-  // Q fragments (A operand, 8 k-steps of 16), as bf16 pairs
+  const bool ok0 = in0 && slot0 >= 0, ok1 = in1 && slot1 >= 0;
+  const uint64_t m00 = ok0 ? mk00 : 0ull, m01 = ok0 ? mk01 : 0ull;
+  const uint64_t m10 = ok1 ? mk10 : 0ull, m11 = ok1 ? mk11 : 0ull;
+  // Q fragments (A operand, 8 k-steps of 16), as bf16 pairs; rows not in use contribute zeros
   uint32_t qh[8][4], ql[8][4];
-  {
-    const float *q0 = q + (size_t)r0 * H + h * DH, *q1 = q + (size_t)r1 * H + h * DH;
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-      const int col = ks * 16 + 2 * t;
-      const float2 a = ok0 ? *reinterpret_cast<const float2 *>(q0 + col) : make_float2(0.f, 0.f);
-      const float2 bq = ok1 ? *reinterpret_cast<const float2 *>(q1 + col) : make_float2(0.f, 0.f);
-      const float2 cq = ok0 ? *reinterpret_cast<const float2 *>(q0 + col + 8) : make_float2(0.f, 0.f);
-      const float2 dq = ok1 ? *reinterpret_cast<const float2 *>(q1 + col + 8) : make_float2(0.f, 0.f);
-      split_pack(a.x, a.y, qh[ks][0], ql[ks][0]);
-      split_pack(bq.x, bq.y, qh[ks][1], ql[ks][1]);
-      split_pack(cq.x, cq.y, qh[ks][2], ql[ks][2]);
-      split_pack(dq.x, dq.y, qh[ks][3], ql[ks][3]);
+  for (int ks = 0; ks < 8; ++ks) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const bool ok = (e & 1) ? ok1 : ok0;
+      split_pack(ok ? qa[ks][e].x : 0.f, ok ? qa[ks][e].y : 0.f, qh[ks][e], ql[ks][e]);
     }
   }
 
@@ -158,19 +167,30 @@ tree_attn_mma_kernel(const float *__restrict__ q, const bf16 *__restrict__ kc, c
     const uint32_t kt = sbase + buf * 2 * TILE_BYTES, vt = kt + TILE_BYTES;
     const int key0 = tile * TILE + kw;
     // ---- S = Q K^T over this warp's 16 keys
-    float s[2][4];
+    // four independent accumulation chains (key group x value/residual part of Q), interleaved
+    float s[2][4], sl[2][4];
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
       s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+      sl[j][0] = sl[j][1] = sl[j][2] = sl[j][3] = 0.f;
+    }
 #pragma unroll
-      for (int kp = 0; kp < 4; ++kp) {
-        uint32_t b0, b1, b2, b3;
-        ldmatrix_x4(kt + tile_off(kw + 8 * j + (lane & 7), 4 * kp + (lane >> 3)), b0, b1, b2, b3);
-        mma_bf16(s[j], qh[2 * kp], b0, b1);
-        mma_bf16(s[j], ql[2 * kp], b0, b1);
-        mma_bf16(s[j], qh[2 * kp + 1], b2, b3);
-        mma_bf16(s[j], ql[2 * kp + 1], b2, b3);
-      }
+    for (int kp = 0; kp < 4; ++kp) {
+      uint32_t ka[4], kb2[4];
+      ldmatrix_x4(kt + tile_off(kw + (lane & 7), 4 * kp + (lane >> 3)), ka[0], ka[1], ka[2], ka[3]);
+      ldmatrix_x4(kt + tile_off(kw + 8 + (lane & 7), 4 * kp + (lane >> 3)), kb2[0], kb2[1], kb2[2], kb2[3]);
+      mma_bf16(s[0], qh[2 * kp], ka[0], ka[1]);
+      mma_bf16(sl[0], ql[2 * kp], ka[0], ka[1]);
+      mma_bf16(s[1], qh[2 * kp], kb2[0], kb2[1]);
+      mma_bf16(sl[1], ql[2 * kp], kb2[0], kb2[1]);
+      mma_bf16(s[0], qh[2 * kp + 1], ka[2], ka[3]);
+      mma_bf16(sl[0], ql[2 * kp + 1], ka[2], ka[3]);
+      mma_bf16(s[1], qh[2 * kp + 1], kb2[2], kb2[3]);
+      mma_bf16(sl[1], ql[2 * kp + 1], kb2[2], kb2[3]);
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      s[j][0] += sl[j][0]; s[j][1] += sl[j][1]; s[j][2] += sl[j][2]; s[j][3] += sl[j][3];
     }
     // ---- mask, online softmax (base 2)
     const bool need_mask = key0 + 16 > ctx;
@@ -224,15 +244,22 @@ tree_attn_mma_kernel(const float *__restrict__ q, const bf16 *__restrict__ kc, c
       for (int j = 0; j < 16; ++j) { o[j][0] *= cr0; o[j][1] *= cr0; o[j][2] *= cr1; o[j][3] *= cr1; }
     }
     // ---- O += P V over this warp's 16 keys, 16 groups of 8 head dims
+    // (all value-part products first, then all residual-part products: 16 independent
+    //  accumulators between two uses of the same one)
+    uint32_t vf[8][4];
+#pragma unroll
+    for (int jp = 0; jp < 8; ++jp)
+      ldmatrix_x4_trans(vt + tile_off(kw + (lane & 7) + 8 * ((lane >> 3) & 1), 2 * jp + (lane >> 4)),
+                        vf[jp][0], vf[jp][1], vf[jp][2], vf[jp][3]);
 #pragma unroll
     for (int jp = 0; jp < 8; ++jp) {
-      uint32_t b0, b1, b2, b3;
-      ldmatrix_x4_trans(vt + tile_off(kw + (lane & 7) + 8 * ((lane >> 3) & 1), 2 * jp + (lane >> 4)),
-                        b0, b1, b2, b3);
-      mma_bf16(o[2 * jp], ph, b0, b1);
-      mma_bf16(o[2 * jp], pl, b0, b1);
-      mma_bf16(o[2 * jp + 1], ph, b2, b3);
-      mma_bf16(o[2 * jp + 1], pl, b2, b3);
+      mma_bf16(o[2 * jp], ph, vf[jp][0], vf[jp][1]);
+      mma_bf16(o[2 * jp + 1], ph, vf[jp][2], vf[jp][3]);
+    }
+#pragma unroll
+    for (int jp = 0; jp < 8; ++jp) {
+      mma_bf16(o[2 * jp], pl, vf[jp][0], vf[jp][1]);
+      mma_bf16(o[2 * jp + 1], pl, vf[jp][2], vf[jp][3]);
     }
     __syncthreads();      // the buffer refilled by the next iteration's load is no longer read
   }

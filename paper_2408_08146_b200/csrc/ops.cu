@@ -165,6 +165,13 @@ row_epilogue_vec_kernel(int mode, float *__restrict__ x, SplitIn P, const T *__r
       ss += o.x * o.x + o.y * o.y + o.z * o.z + o.w * o.w;
     }
   }
+  // the gains are fetched before the block-wide reduction so that their latency hides behind it
+  float4 gg[VPT];
+#pragma unroll
+  for (int k = 0; k < VPT; ++k) {
+    const int c = (threadIdx.x + k * blockDim.x) * 4;
+    gg[k] = (g != nullptr && c < H) ? load4<T>(g + c) : make_float4(1.f, 1.f, 1.f, 1.f);
+  }
   float inv = 1.f;
   if (g != nullptr) inv = rsqrtf(block_sum(ss, red) / (float)H + eps);
 #pragma unroll
@@ -173,8 +180,7 @@ row_epilogue_vec_kernel(int mode, float *__restrict__ x, SplitIn P, const T *__r
     if (c < H) {
       float4 n = v[k];
       if (g != nullptr) {
-        const float4 gg = load4<T>(g + c);
-        n = make_float4(n.x * inv * gg.x, n.y * inv * gg.y, n.z * inv * gg.z, n.w * inv * gg.w);
+        n = make_float4(n.x * inv * gg[k].x, n.y * inv * gg[k].y, n.z * inv * gg[k].z, n.w * inv * gg[k].w);
       }
       if (xn != nullptr) store_operand4(xn, xn_lo, (size_t)r * H + c, n);
       if (out_f32 != nullptr) *reinterpret_cast<float4 *>(out_f32 + (size_t)r * H + c) = n;
