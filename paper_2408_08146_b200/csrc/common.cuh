@@ -35,16 +35,28 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
-// A matrix given as the sum of `n` partial matrices `stride` floats apart (split-K results).
+// A matrix given as the sum of partial matrices `stride` floats apart (split-K results).
+// Classic split-K: every column has `n` partials.  Stream-K (sk_ctas > 0): column c belongs to
+// weight tile c / 128, whose K-blocks were dealt to the CTAs owning units
+// [tile * sk_kb, (tile + 1) * sk_kb); it has one partial per such CTA, in slots 0, 1, ...
 struct SplitIn {
   const float *p;
   int n;
   size_t stride;
   int ld;
+  unsigned sk_ctas, sk_units, sk_kb;
+  __device__ __forceinline__ int count(int c) const {
+    if (sk_ctas == 0) return n;
+    const unsigned u0 = (unsigned)(c >> 7) * sk_kb;
+    const unsigned first = ((u0 + 1u) * sk_ctas - 1u) / sk_units;
+    const unsigned last = ((u0 + sk_kb) * sk_ctas - 1u) / sk_units;
+    return (int)(last - first) + 1;
+  }
   __device__ __forceinline__ float at(int r, int c) const {
     const float *q = p + (size_t)r * ld + c;
+    const int k = count(c);
     float v = q[0];
-    for (int s = 1; s < n; ++s) v += q[(size_t)s * stride];
+    for (int s = 1; s < k; ++s) v += q[(size_t)s * stride];
     return v;
   }
 };
@@ -137,8 +149,11 @@ cudaError_t gemm_simt(Launch L, int dtype, Operand X, GemmMats m, int K_in, int 
 int tc_init_driver(char *err, size_t errlen);   // 0 on success
 bool tc_supported(const GemmMats &m, int K_in);
 int tc_default_split(int n_tiles, int kblocks, int tokens);
+// split >= 1: classic split-K; split == 0: automatic (stream-K where it applies).  `max_slots`
+// bounds the partial matrices written; *out describes them for the consumer.
 cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in, int R,
-                    float *Y, int ldy, int split, size_t split_stride, int *status);
+                    float *Y, int ldy, int split, size_t split_stride, int *status, int max_slots,
+                    SplitIn *out);
 
 // tree.cu
 struct TreeBufs {

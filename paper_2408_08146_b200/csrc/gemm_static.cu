@@ -49,16 +49,16 @@ int koala_gemm_bf16_static(const void *X, const void *X_lo, const void *W, float
   Operand Xo{const_cast<void *>(X), const_cast<void *>(X_lo)};
   const int rows_alloc = koala_gemm_x_rows(M, X_lo != nullptr);
   if (split == 1)
-    return gemm_tc(L, Xo, rows_alloc, m, K_in, M, Y, ldy, 1, 0, device_status) == cudaSuccess ? KOALA_OK
+    return gemm_tc(L, Xo, rows_alloc, m, K_in, M, Y, ldy, 1, 0, device_status, 1, nullptr) == cudaSuccess ? KOALA_OK
                                                                                               : KOALA_E_CUDA;
   const size_t stride = (size_t)M * N_out;
   if ((size_t)split * stride > STATIC_SCRATCH_FLOATS) return KOALA_E_CAPACITY;
   float *scratch = g_scratch_ptr[dev];
   // every partial element that is read below is written by exactly one CTA of this launch, so the
   // previous call's contents need no clearing
-  if (gemm_tc(L, Xo, rows_alloc, m, K_in, M, scratch, N_out, split, stride, device_status) != cudaSuccess)
+  SplitIn s;
+  if (gemm_tc(L, Xo, rows_alloc, m, K_in, M, scratch, N_out, split, stride, device_status, split, &s) != cudaSuccess)
     return KOALA_E_CUDA;
-  SplitIn s{scratch, split, stride, N_out};
   return reduce_splits(L, s, Y, ldy, M, N_out) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
 }
 

@@ -120,16 +120,24 @@ struct TcParams {
   int bn;             // MMA N = rows of the activation tile in shared memory, multiple of 16, <= 256
   int tt;             // tokens per tile: bn, or bn / 2 when the activations are a hi/lo pair
   int pair;           // 1: hi/lo pair
-  int ztiles;         // token tiles (fastest-varying part of blockIdx.x)
-  int tmem_cols;      // power of two >= max(32, bn)
+  int ztiles;         // token tiles (classic mode; fastest-varying part of blockIdx.x)
+  int tmem_cols;      // power of two >= max(32, bn), per accumulator buffer
+  int nbuf;           // accumulator buffers in tensor memory (2 when they fit in 256 columns)
   int tiles0, tiles1; // weight tiles of matrix 0 and of matrices 0+1 (cumulative)
   int n0, n1, n2;     // rows of each matrix
   int kblocks;        // K_in / 64
-  int split;          // CTAs along K
+  int split;          // classic mode: CTAs along K (grid.y)
+  int sk_ctas;        // stream-K mode (> 0): the grid's CTAs share all (tile, K-block) units evenly
+  unsigned sk_units;  // tiles * kblocks
   size_t split_stride;
   int stages;
   int *status;
 };
+
+// CTA that owns unit u when `units` units are dealt to `ctas` CTAs as [g*units/ctas, (g+1)*units/ctas)
+__device__ __forceinline__ unsigned sk_owner(unsigned u, unsigned ctas, unsigned units) {
+  return ((u + 1u) * ctas - 1u) / units;
+}
 
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
@@ -138,7 +146,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   extern __shared__ unsigned char smem_raw[];
   __shared__ uint64_t full_bar[MAX_STAGES];
   __shared__ uint64_t empty_bar[MAX_STAGES];
-  __shared__ uint64_t accum_bar;
+  __shared__ uint64_t acc_full[2];      // accumulator buffer complete (MMA -> epilogue)
+  __shared__ uint64_t acc_empty[2];     // accumulator buffer drained (epilogue -> MMA)
   __shared__ uint32_t tmem_base_slot;
   __shared__ int s_error;
 
@@ -146,35 +155,39 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char *tiles = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
   const int x_stage_bytes = P.bn * BK * 2;
-  const int stage_bytes = W_STAGE_BYTES + x_stage_bytes;   // both multiples of 1024 (bn % 16 == 0 -> x multiple of 2048)
+  const int stage_bytes = W_STAGE_BYTES + x_stage_bytes;   // both multiples of 1024
+  const int KB = P.kblocks;
 
-  // which matrix / which rows
-  int tile = blockIdx.x / P.ztiles;
-  const int ztile = blockIdx.x % P.ztiles;
-  const CUtensorMap *tmW = &tmW0;
-  int col_off = 0, n_rows = P.n0;
-  if (tile >= P.tiles1) { tmW = &tmW2; tile -= P.tiles1; col_off = P.n0 + P.n1; n_rows = P.n2; }
-  else if (tile >= P.tiles0) { tmW = &tmW1; tile -= P.tiles0; col_off = P.n0; n_rows = P.n1; }
-  const int row0 = tile * BM;
-  const int tok0 = ztile * P.tt;
-  // K range of this split
-  const int kb_lo = (int)(((long long)P.kblocks * blockIdx.y) / P.split);
-  const int kb_hi = (int)(((long long)P.kblocks * (blockIdx.y + 1)) / P.split);
-  const int nkb = kb_hi - kb_lo;
+  // this CTA's run of (tile, K-block) units, tile-major; a run may cross tile boundaries (stream-K)
+  unsigned u_lo, u_hi;
+  int tok0 = 0;
+  if (P.sk_ctas > 0) {
+    u_lo = (unsigned)(((unsigned long long)blockIdx.x * P.sk_units) / (unsigned)P.sk_ctas);
+    u_hi = (unsigned)(((unsigned long long)(blockIdx.x + 1) * P.sk_units) / (unsigned)P.sk_ctas);
+  } else {
+    const int tile = blockIdx.x / P.ztiles;
+    tok0 = (blockIdx.x % P.ztiles) * P.tt;
+    u_lo = (unsigned)(tile * KB + (int)(((long long)KB * blockIdx.y) / P.split));
+    u_hi = (unsigned)(tile * KB + (int)(((long long)KB * (blockIdx.y + 1)) / P.split));
+  }
+  const int n_units = (int)(u_hi - u_lo);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < P.stages; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    mbar_init(&accum_bar, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&acc_full[i], 1);
+      mbar_init(&acc_empty[i], 4);       // one arrival per epilogue warp
+    }
     s_error = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)P.tmem_cols)
+                 ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)(P.tmem_cols * P.nbuf))
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -184,42 +197,62 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   const uint32_t tmem_acc = tmem_base_slot;
   pdl_launch_dependents();
 
+  // weight tensor map and first row of a tile
+  auto tile_map = [&](int tile, int &row0) -> const CUtensorMap * {
+    if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * BM; return &tmW2; }
+    if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * BM; return &tmW1; }
+    row0 = tile * BM;
+    return &tmW0;
+  };
+
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(tmW) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW0) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
       if (P.pair) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmXlo) : "memory");
-      const int pre = nkb < P.stages ? nkb : P.stages;
+      const int pre = n_units < P.stages ? n_units : P.stages;
       // weights first: they do not depend on the kernel before this one
       for (int it = 0; it < pre; ++it) {
+        const unsigned u = u_lo + it;
+        int row0;
+        const CUtensorMap *tmW = tile_map((int)(u / KB), row0);
         mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
-        tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, (kb_lo + it) * BK, row0);
+        tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, (int)(u % KB) * BK, row0);
       }
       // and a few more of this CTA's weight tiles are requested into L2 while the producer of X
       // runs (bounded, so that all CTAs together stay well inside the L2)
-      const int ahead = nkb < pre + L2_AHEAD ? nkb : pre + L2_AHEAD;
-      for (int it = pre; it < ahead; ++it)
+      const int ahead = n_units < pre + L2_AHEAD ? n_units : pre + L2_AHEAD;
+      for (int it = pre; it < ahead; ++it) {
+        const unsigned u = u_lo + it;
+        int row0;
+        const CUtensorMap *tmW = tile_map((int)(u / KB), row0);
         asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
-                     ::"l"(tmW), "r"((kb_lo + it) * BK), "r"(row0) : "memory");
+                     ::"l"(tmW), "r"((int)(u % KB) * BK), "r"(row0) : "memory");
+      }
       pdl_wait();
       const int lo_off = P.tt * BK * 2;          // the lo rows follow the hi rows of the tile
       for (int it = 0; it < pre; ++it) {
+        const int kx = (int)((u_lo + it) % KB) * BK;
         unsigned char *xd = tiles + (size_t)it * stage_bytes + W_STAGE_BYTES;
-        tma_load_2d(&tmX, &full_bar[it], xd, (kb_lo + it) * BK, tok0);
-        if (P.pair) tma_load_2d(&tmXlo, &full_bar[it], xd + lo_off, (kb_lo + it) * BK, tok0);
+        tma_load_2d(&tmX, &full_bar[it], xd, kx, tok0);
+        if (P.pair) tma_load_2d(&tmXlo, &full_bar[it], xd + lo_off, kx, tok0);
       }
       bool ok = true;
-      for (int it = pre; it < nkb && ok; ++it) {
+      for (int it = pre; it < n_units && ok; ++it) {
         const int s = it % P.stages;
         const uint32_t ph = (uint32_t)(it / P.stages) & 1u;
         ok = mbar_wait(&empty_bar[s], ph ^ 1u);
         if (!ok) break;
+        const unsigned u = u_lo + it;
+        int row0;
+        const CUtensorMap *tmW = tile_map((int)(u / KB), row0);
+        const int kx = (int)(u % KB) * BK;
         mbar_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
         unsigned char *dst = tiles + (size_t)s * stage_bytes;
-        tma_load_2d(tmW, &full_bar[s], dst, (kb_lo + it) * BK, row0);
-        tma_load_2d(&tmX, &full_bar[s], dst + W_STAGE_BYTES, (kb_lo + it) * BK, tok0);
-        if (P.pair) tma_load_2d(&tmXlo, &full_bar[s], dst + W_STAGE_BYTES + lo_off, (kb_lo + it) * BK, tok0);
+        tma_load_2d(tmW, &full_bar[s], dst, kx, row0);
+        tma_load_2d(&tmX, &full_bar[s], dst + W_STAGE_BYTES, kx, tok0);
+        if (P.pair) tma_load_2d(&tmXlo, &full_bar[s], dst + W_STAGE_BYTES + lo_off, kx, tok0);
       }
       if (!ok) {
         atomicExch(&s_error, 1);
@@ -234,7 +267,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.bn >> 3) << 17) |
                              ((uint32_t)(BM >> 4) << 24);
       bool ok = true;
-      for (int it = 0; it < nkb; ++it) {
+      int seg = 0;                        // segment = run of units inside one tile
+      bool seg_start = true;
+      for (int it = 0; it < n_units; ++it) {
+        const unsigned u = u_lo + it;
+        const int buf = seg % P.nbuf;
+        if (seg_start && seg >= P.nbuf) {
+          // the accumulator buffer must have been drained by the epilogue of segment seg - nbuf
+          ok = mbar_wait(&acc_empty[buf], (uint32_t)((seg / P.nbuf) - 1) & 1u);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        }
         const int s = it % P.stages;
         const uint32_t ph = (uint32_t)(it / P.stages) & 1u;
         ok = mbar_wait(&full_bar[s], ph);
@@ -243,50 +286,78 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         const uint32_t wa = smem_u32(tiles + (size_t)s * stage_bytes);
         const uint64_t da = smem_desc_sw128(wa);
         const uint64_t db = smem_desc_sw128(wa + W_STAGE_BYTES);
+        const uint32_t dacc = tmem_acc + (uint32_t)(buf * P.tmem_cols);
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; ++k) {
           // advance 32 bytes (16 bf16) inside the swizzled row: +2 in the 16-byte address field
-          umma_bf16(tmem_acc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
-                    (it > 0 || k > 0) ? 1u : 0u);
+          umma_bf16(dacc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
+                    (!seg_start || k > 0) ? 1u : 0u);
         }
         umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
+        const bool seg_end = (u % KB) == (unsigned)(KB - 1) || it == n_units - 1;
+        if (seg_end) {
+          umma_commit(&acc_full[buf]);   // this segment's accumulator is complete
+          ++seg;
+        }
+        seg_start = seg_end;
       }
-      if (ok) umma_commit(&accum_bar);   // accumulator complete
-      else atomicExch(&s_error, 1);
+      if (!ok) atomicExch(&s_error, 1);
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quarter = warp & 3;        // the 32 tensor-memory lanes this warp may read
     pdl_wait();                          // the output buffer may still be read by the previous kernel
-    bool ok = mbar_wait(&accum_bar, 0);
-    if (!ok) atomicExch(&s_error, 1);
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const int feat = row0 + quarter * 32 + lane;
-    float *Yp = P.Y + (size_t)blockIdx.y * P.split_stride + col_off + feat;
-    if (ok) {
+    bool ok = true;
+    int seg = 0;
+    unsigned u = u_lo;
+    while (u < u_hi && ok) {
+      const int tile = (int)(u / KB);
+      unsigned seg_hi = (unsigned)(tile + 1) * KB;
+      if (seg_hi > u_hi) seg_hi = u_hi;
+      const int buf = seg % P.nbuf;
+      ok = mbar_wait(&acc_full[buf], (uint32_t)(seg / P.nbuf) & 1u);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      int row0, col_off = 0, n_rows = P.n0;
+      if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * BM; col_off = P.n0 + P.n1; n_rows = P.n2; }
+      else if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * BM; col_off = P.n0; n_rows = P.n1; }
+      else row0 = tile * BM;
+      // which partial-sum slot: classic = the split index; stream-K = rank among the tile's contributors
+      int slot = blockIdx.y;
+      if (P.sk_ctas > 0)
+        slot = (int)blockIdx.x - (int)sk_owner((unsigned)tile * KB, (unsigned)P.sk_ctas, P.sk_units);
+      const int feat = row0 + quarter * 32 + lane;
+      float *Yp = P.Y + (size_t)slot * P.split_stride + col_off + feat;
+      const uint32_t lane_base = tmem_acc + (uint32_t)(buf * P.tmem_cols) + ((uint32_t)(quarter * 32) << 16);
       for (int c0 = 0; c0 < P.tt; c0 += 16) {
-        uint32_t v[16], u[16];
-        const uint32_t lane_base = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+        uint32_t v[16], w[16];
         tmem_ld16(lane_base + (uint32_t)c0, v);
-        if (P.pair) tmem_ld16(lane_base + (uint32_t)(P.tt + c0), u);
+        if (P.pair) tmem_ld16(lane_base + (uint32_t)(P.tt + c0), w);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (feat < n_rows) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int t = tok0 + c0 + j;
             float r = __uint_as_float(v[j]);
-            if (P.pair) r += __uint_as_float(u[j]);
+            if (P.pair) r += __uint_as_float(w[j]);
             if (t < P.R) Yp[(size_t)t * P.ldy] = r;
           }
         }
       }
+      // hand the accumulator buffer back to the MMA issuer
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&acc_empty[buf])) : "memory");
+      ++seg;
+      u = seg_hi;
     }
+    if (!ok) atomicExch(&s_error, 1);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
-                 ::"r"(tmem_acc), "r"((uint32_t)P.tmem_cols)
+                 ::"r"(tmem_acc), "r"((uint32_t)(P.tmem_cols * P.nbuf))
                  : "memory");
   }
   if (threadIdx.x == 0 && s_error && P.status) atomicMax(P.status, E_TIMEOUT);
@@ -384,8 +455,34 @@ int tc_default_split(int n_tiles, int kblocks, int tokens) {
   return s < 1 ? 1 : s;
 }
 
+// Stream-K plan: how many CTAs share the (tile, K-block) units.  At most two per SM, at least 8
+// units per CTA, at most `max_slots` contributors to any tile, and the fp32 partial sums written
+// and re-read stay below about half of the weight bytes.  Returns 0 when the classic per-tile
+// decomposition is at least as good (one contributor per tile already fills the machine).
+int tc_streamk_ctas(int n_tiles, int kblocks, int tokens, int max_slots, int *slots_out) {
+  const long long units = (long long)n_tiles * kblocks;
+  long long g = 2LL * g_num_sms;
+  if (g > units / 8) g = units / 8;
+  if (g < 1) g = 1;
+  // average contributors per tile = kblocks * g / units; bound it by the traffic rule
+  const long long by_traffic = (long long)(kblocks * 64) / (8LL * (tokens > 0 ? tokens : 1));
+  const long long avg_cap = by_traffic < 1 ? 1 : by_traffic;
+  if ((long long)kblocks * g > avg_cap * units) g = avg_cap * units / kblocks;
+  if (g_tune_max_split > 0 && (long long)kblocks * g > (long long)g_tune_max_split * units)
+    g = (long long)g_tune_max_split * units / kblocks;
+  if (g < 1) g = 1;
+  auto slots_of = [&](long long gg) {
+    const long long per = units / gg;                 // smallest run length
+    return (int)((kblocks + per - 1) / per) + ((units % gg) || (kblocks % per) ? 1 : 0);
+  };
+  while (g > 1 && slots_of(g) > max_slots) --g;
+  *slots_out = slots_of(g);
+  return (int)g;
+}
+
 cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in, int R,
-                    float *Y, int ldy, int split, size_t split_stride, int *status) {
+                    float *Y, int ldy, int split, size_t split_stride, int *status, int max_slots,
+                    SplitIn *out) {
   if (!tc_supported(m, K_in) || R < 1 || ((uintptr_t)X.hi & 15u) || ((uintptr_t)X.lo & 15u))
     return cudaErrorInvalidValue;
   TcParams P;
@@ -412,17 +509,34 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   const int t0 = (m.n_out[0] + BM - 1) / BM;
   const int t1 = m.n > 1 ? (m.n_out[1] + BM - 1) / BM : 0;
   const int t2 = m.n > 2 ? (m.n_out[2] + BM - 1) / BM : 0;
+  const int n_tiles = t0 + t1 + t2;
   P.tiles0 = t0;
   P.tiles1 = t0 + t1;
   P.n0 = m.n_out[0];
   P.n1 = m.n > 1 ? m.n_out[1] : 0;
   P.n2 = m.n > 2 ? m.n_out[2] : 0;
   P.kblocks = K_in / BK;
-  if (split < 1) split = 1;
-  if (split > P.kblocks) split = P.kblocks;
-  P.split = split;
+  // stream-K (split == 0): needs a single token tile and 128-row-aligned matrices, so that a
+  // column's tile (and with it the number of partial sums to add) follows from the column index
+  bool sk = split == 0 && ztiles == 1 && max_slots >= 2 && out != nullptr;
+  for (int i = 0; i < m.n && sk; ++i) sk = (m.n_out[i] % BM) == 0;
+  int sk_ctas = 0, sk_slots = 1;
+  if (sk) {
+    sk_ctas = tc_streamk_ctas(n_tiles, P.kblocks, R, max_slots, &sk_slots);
+    if (sk_ctas <= n_tiles) sk = false;         // nothing to share: one CTA per tile is the same thing
+  }
+  if (!sk) {
+    sk_ctas = 0;
+    if (split < 1) split = tc_default_split(n_tiles, P.kblocks, R);
+    if (split > P.kblocks) split = P.kblocks;
+    if (max_slots > 0 && split > max_slots) split = max_slots;
+  }
+  P.split = sk ? 1 : split;
+  P.sk_ctas = sk_ctas;
+  P.sk_units = (unsigned)((long long)n_tiles * P.kblocks);
   P.split_stride = split_stride;
   P.status = status;
+  P.nbuf = (sk && 2 * cols <= 256) ? 2 : 1;
   const int stage_bytes = W_STAGE_BYTES + bn * BK * 2;
   int stages = (g_smem_optin - 2048) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -441,8 +555,12 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   }
   if (!get_map(X.hi, x_rows_alloc, K_in, tt, &mx)) return cudaErrorInvalidValue;
   if (!get_map(pair ? X.lo : X.hi, x_rows_alloc, K_in, tt, &mxlo)) return cudaErrorInvalidValue;
-  dim3 grid((t0 + t1 + t2) * ztiles, split, 1);
+  dim3 grid = sk ? dim3(sk_ctas, 1, 1) : dim3(n_tiles * ztiles, split, 1);
   const size_t smem = (size_t)stages * stage_bytes + 1024;
+  if (out) {
+    *out = SplitIn{Y, sk ? sk_slots : split, split_stride, ldy, sk ? (unsigned)sk_ctas : 0u, P.sk_units,
+                   (unsigned)P.kblocks};
+  }
   return launch_k(gemm_tc_kernel, grid, dim3(THREADS), smem, L.st, L.pdl, mw[0], mw[1], mw[2], mx, mxlo, P);
 }
 

@@ -39,7 +39,7 @@ struct Carver {
   }
 };
 
-constexpr int MAX_SPLIT = 8;
+constexpr int MAX_SPLIT = 12;     // partial-sum matrices the workspace holds per GEMM
 
 }  // namespace
 
@@ -253,20 +253,17 @@ int do_gemm(koala_ctx *c, Operand X, int K_in, GemmMats m, int R, float *direct,
   const int ld = direct ? ld_direct : ncols;
   const uint64_t wbytes = (uint64_t)ncols * K_in * c->esz;
   if (c->use_tc && c->cfg.dtype == KOALA_BF16 && tc_supported(m, K_in)) {
-    int tiles = 0;
-    for (int i = 0; i < m.n; ++i) tiles += (m.n_out[i] + 127) / 128;
-    int split = direct ? 1 : tc_default_split(tiles, K_in / 64, R);
-    if (split > MAX_SPLIT) split = MAX_SPLIT;
     const size_t stride = (size_t)c->Mp * ld;
     const int tb = time_begin(c, KOALA_CLS_GEMM_TC, wbytes);
-    CU_TRY(gemm_tc(LN(c), X, c->Mp, m, K_in, R, Y, ld, split, stride, c->status));
+    SplitIn res;
+    CU_TRY(gemm_tc(LN(c), X, c->Mp, m, K_in, R, Y, ld, direct ? 1 : 0, stride, c->status, MAX_SPLIT, &res));
     time_end(c, tb);
-    if (out) *out = SplitIn{Y, split, stride, ld};
+    if (out) *out = res;
   } else {
     const int tb = time_begin(c, KOALA_CLS_GEMM_SIMT, wbytes);
     CU_TRY(gemm_simt(LN(c), c->cfg.dtype, X, m, K_in, R, Y, ld));
     time_end(c, tb);
-    if (out) *out = SplitIn{Y, 1, 0, ld};
+    if (out) *out = SplitIn{Y, 1, 0, ld, 0u, 0u, 0u};
   }
   return KOALA_OK;
 }
@@ -708,20 +705,19 @@ int koala_gemm_bf16(const void *X, const void *X_lo, const void *W, float *Y, in
   char e[160];
   if (tc_init_driver(e, sizeof(e)) != 0) return KOALA_E_CUDA;
   if (!tc_supported(m, K_in)) return KOALA_E_UNSUPPORTED;
-  int split = split_k > 0 ? split_k : tc_default_split((N_out + 127) / 128, K_in / 64, M);
-  if (split > MAX_SPLIT) split = MAX_SPLIT;
-  if (split > K_in / 64) split = K_in / 64;
-  // X must hold a whole token tile: the caller's buffer has M rows, rounded up by the map's
-  // out-of-bounds zero fill
+  if (split_k > MAX_SPLIT) split_k = MAX_SPLIT;
+  if (split_k < 0) split_k = 0;
+  // X must hold whole token tiles (koala_gemm_x_rows)
   const int rows_alloc = koala_gemm_x_rows(M, X_lo != nullptr);
-  if (split == 1) {
-    return gemm_tc(L, Xo, rows_alloc, m, K_in, M, Y, ldy, 1, 0, device_status) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
-  }
+  if (split_k == 1)
+    return gemm_tc(L, Xo, rows_alloc, m, K_in, M, Y, ldy, 1, 0, device_status, 1, nullptr) == cudaSuccess
+               ? KOALA_OK : KOALA_E_CUDA;
   const size_t stride = (size_t)M * N_out;
-  if (!scratch || scratch_bytes < (size_t)split * stride * sizeof(float)) return KOALA_E_CAPACITY;
-  if (gemm_tc(L, Xo, rows_alloc, m, K_in, M, (float *)scratch, N_out, split, stride, device_status) != cudaSuccess)
+  if (!scratch || scratch_bytes < (size_t)MAX_SPLIT * stride * sizeof(float)) return KOALA_E_CAPACITY;
+  SplitIn s;
+  if (gemm_tc(L, Xo, rows_alloc, m, K_in, M, (float *)scratch, N_out, split_k, stride, device_status, MAX_SPLIT,
+              &s) != cudaSuccess)
     return KOALA_E_CUDA;
-  SplitIn s{(const float *)scratch, split, stride, N_out};
   return reduce_splits(L, s, Y, ldy, M, N_out) == cudaSuccess ? KOALA_OK : KOALA_E_CUDA;
 }
 

@@ -95,7 +95,8 @@ __global__ void row_epilogue_kernel(int mode, float *__restrict__ x, SplitIn P,
 __device__ __forceinline__ float4 split_sum4(const SplitIn &P, int r, int c) {
   const float *q = P.p + (size_t)r * P.ld + c;
   float4 v = *reinterpret_cast<const float4 *>(q);
-  for (int s = 1; s < P.n; ++s) {
+  const int k = P.count(c);
+  for (int s = 1; s < k; ++s) {
     const float4 u = *reinterpret_cast<const float4 *>(q + (size_t)s * P.stride);
     v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
   }
@@ -265,7 +266,8 @@ __global__ void rope_kv_kernel(SplitIn qkv, RowPlan plan, float *__restrict__ q_
 __device__ __forceinline__ float2 split_sum2(const SplitIn &P, int r, int c) {
   const float *q = P.p + (size_t)r * P.ld + c;
   float2 v = *reinterpret_cast<const float2 *>(q);
-  for (int s = 1; s < P.n; ++s) {
+  const int k = P.count(c);
+  for (int s = 1; s < k; ++s) {
     const float2 u = *reinterpret_cast<const float2 *>(q + (size_t)s * P.stride);
     v.x += u.x; v.y += u.y;
   }
