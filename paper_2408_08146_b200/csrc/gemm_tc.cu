@@ -520,6 +520,13 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   // column's tile (and with it the number of partial sums to add) follows from the column index
   bool sk = split == 0 && ztiles == 1 && max_slots >= 2 && out != nullptr;
   for (int i = 0; i < m.n && sk; ++i) sk = (m.n_out[i] % BM) == 0;
+  // stream-K pays off where the per-tile decomposition cannot be split further and leaves the SMs
+  // unevenly loaded (more tiles than SMs, not a whole number of two-per-SM waves); elsewhere
+  // classic split-K gives the same balance with fewer partial sums per tile
+  if (sk) {
+    const int classic = tc_default_split(n_tiles, P.kblocks, R);
+    sk = classic == 1 && n_tiles > g_num_sms && (n_tiles % (2 * g_num_sms)) != 0;
+  }
   int sk_ctas = 0, sk_slots = 1;
   if (sk) {
     sk_ctas = tc_streamk_ctas(n_tiles, P.kblocks, R, max_slots, &sk_slots);
