@@ -212,7 +212,8 @@ int koala_timing_read(koala_ctx *ctx, koala_timing *out);
 
 /* Process-wide tuning of the tensor-core matrix multiply (for sweeps; the defaults are chosen
  * for B200): key 1 = shared-memory pipeline stages per CTA (0 = as many as fit, at most 8);
- * key 2 = upper bound on the automatic split-K factor (0 = default). */
+ * key 2 = upper bound on the automatic split-K factor (0 = default); key 3 = 1 switches stream-K
+ * off (every CTA stays inside one weight tile). */
 void koala_set_tuning(int key, int value);
 
 /* Kernels launched by the library in this process so far (all contexts). */

@@ -208,56 +208,56 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW0) : "memory");
+      // (tile, K-block) of the next unit, advanced incrementally
+      int tile = (int)(u_lo / KB), kb = (int)(u_lo % KB), row0;
+      const CUtensorMap *tmW = tile_map(tile, row0);
+      asm volatile("prefetch.tensormap [%0];" ::"l"(tmW) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
       if (P.pair) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmXlo) : "memory");
       const int pre = n_units < P.stages ? n_units : P.stages;
-      // weights first: they do not depend on the kernel before this one
-      for (int it = 0; it < pre; ++it) {
-        const unsigned u = u_lo + it;
-        int row0;
-        const CUtensorMap *tmW = tile_map((int)(u / KB), row0);
-        mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
-        tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, (int)(u % KB) * BK, row0);
-      }
-      // and a few more of this CTA's weight tiles are requested into L2 while the producer of X
-      // runs (bounded, so that all CTAs together stay well inside the L2)
       const int ahead = n_units < pre + L2_AHEAD ? n_units : pre + L2_AHEAD;
-      for (int it = pre; it < ahead; ++it) {
-        const unsigned u = u_lo + it;
-        int row0;
-        const CUtensorMap *tmW = tile_map((int)(u / KB), row0);
-        asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
-                     ::"l"(tmW), "r"((int)(u % KB) * BK), "r"(row0) : "memory");
+      // weights first: they do not depend on the kernel before this one; a few more of this CTA's
+      // weight tiles are requested into L2 while the producer of X runs (bounded, so that all CTAs
+      // together stay well inside the L2)
+      for (int it = 0; it < ahead; ++it) {
+        if (it < pre) {
+          mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
+          tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, kb * BK, row0);
+        } else {
+          asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+                       ::"l"(tmW), "r"(kb * BK), "r"(row0) : "memory");
+        }
+        if (++kb == KB) { kb = 0; ++tile; tmW = tile_map(tile, row0); }
       }
       pdl_wait();
       const int lo_off = P.tt * BK * 2;          // the lo rows follow the hi rows of the tile
+      tile = (int)(u_lo / KB);
+      kb = (int)(u_lo % KB);
+      tmW = tile_map(tile, row0);
       for (int it = 0; it < pre; ++it) {
-        const int kx = (int)((u_lo + it) % KB) * BK;
         unsigned char *xd = tiles + (size_t)it * stage_bytes + W_STAGE_BYTES;
-        tma_load_2d(&tmX, &full_bar[it], xd, kx, tok0);
-        if (P.pair) tma_load_2d(&tmXlo, &full_bar[it], xd + lo_off, kx, tok0);
+        tma_load_2d(&tmX, &full_bar[it], xd, kb * BK, tok0);
+        if (P.pair) tma_load_2d(&tmXlo, &full_bar[it], xd + lo_off, kb * BK, tok0);
+        if (++kb == KB) { kb = 0; ++tile; tmW = tile_map(tile, row0); }
       }
       bool ok = true;
-      for (int it = pre; it < n_units && ok; ++it) {
-        const int s = it % P.stages;
-        const uint32_t ph = (uint32_t)(it / P.stages) & 1u;
+      int s = pre % P.stages;
+      uint32_t ph = (uint32_t)(pre / P.stages) & 1u;
+      for (int it = pre; it < n_units; ++it) {
         ok = mbar_wait(&empty_bar[s], ph ^ 1u);
         if (!ok) break;
-        const unsigned u = u_lo + it;
-        int row0;
-        const CUtensorMap *tmW = tile_map((int)(u / KB), row0);
-        const int kx = (int)(u % KB) * BK;
         mbar_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
         unsigned char *dst = tiles + (size_t)s * stage_bytes;
-        tma_load_2d(tmW, &full_bar[s], dst, kx, row0);
-        tma_load_2d(&tmX, &full_bar[s], dst + W_STAGE_BYTES, kx, tok0);
-        if (P.pair) tma_load_2d(&tmXlo, &full_bar[s], dst + W_STAGE_BYTES + lo_off, kx, tok0);
+        tma_load_2d(tmW, &full_bar[s], dst, kb * BK, row0);
+        tma_load_2d(&tmX, &full_bar[s], dst + W_STAGE_BYTES, kb * BK, tok0);
+        if (P.pair) tma_load_2d(&tmXlo, &full_bar[s], dst + W_STAGE_BYTES + lo_off, kb * BK, tok0);
+        if (++kb == KB) { kb = 0; ++tile; tmW = tile_map(tile, row0); }
+        if (++s == P.stages) { s = 0; ph ^= 1u; }
       }
       if (!ok) {
         atomicExch(&s_error, 1);
         // let the copies already requested land before the block's memory goes away
-        for (int s = 0; s < P.stages; ++s) (void)mbar_wait(&full_bar[s], 0);
+        for (int q = 0; q < P.stages; ++q) (void)mbar_wait(&full_bar[q], 0);
       }
     }
   } else if (warp == 1) {
@@ -269,17 +269,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       bool ok = true;
       int seg = 0;                        // segment = run of units inside one tile
       bool seg_start = true;
+      int kb = (int)(u_lo % KB), s = 0, buf = 0;
+      uint32_t ph = 0;
       for (int it = 0; it < n_units; ++it) {
-        const unsigned u = u_lo + it;
-        const int buf = seg % P.nbuf;
         if (seg_start && seg >= P.nbuf) {
           // the accumulator buffer must have been drained by the epilogue of segment seg - nbuf
           ok = mbar_wait(&acc_empty[buf], (uint32_t)((seg / P.nbuf) - 1) & 1u);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         }
-        const int s = it % P.stages;
-        const uint32_t ph = (uint32_t)(it / P.stages) & 1u;
         ok = mbar_wait(&full_bar[s], ph);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -294,12 +292,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                     (!seg_start || k > 0) ? 1u : 0u);
         }
         umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
-        const bool seg_end = (u % KB) == (unsigned)(KB - 1) || it == n_units - 1;
+        const bool seg_end = (kb == KB - 1) || it == n_units - 1;
         if (seg_end) {
           umma_commit(&acc_full[buf]);   // this segment's accumulator is complete
           ++seg;
+          buf = (P.nbuf == 2) ? (buf ^ 1) : 0;
         }
         seg_start = seg_end;
+        if (++kb == KB) kb = 0;
+        if (++s == P.stages) { s = 0; ph ^= 1u; }
       }
       if (!ok) atomicExch(&s_error, 1);
     }
@@ -375,6 +376,7 @@ int g_smem_optin = 0;
 int g_num_sms = 148;
 int g_tune_stages = 0;      // 0 = as many as fit (at most 8)
 int g_tune_max_split = 0;   // 0 = default rule
+int g_tune_no_streamk = 0;  // 1 = always the per-tile decomposition
 
 bool get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out) {
   std::lock_guard<std::mutex> lock(g_mu);
@@ -427,6 +429,7 @@ int tc_init_driver(char *err, size_t errlen) {
 void tc_set_tuning(int key, int value) {
   if (key == 1) g_tune_stages = value;
   if (key == 2) g_tune_max_split = value;
+  if (key == 3) g_tune_no_streamk = value;
 }
 
 void tc_forget_maps() {
@@ -451,6 +454,7 @@ int tc_default_split(int n_tiles, int kblocks, int tokens) {
   const int by_traffic = (kblocks * 64) / (8 * (tokens > 0 ? tokens : 1));
   if (s > by_k) s = by_k;
   if (s > by_traffic) s = by_traffic;
+  if (s > 8) s = 8;
   if (g_tune_max_split > 0 && s > g_tune_max_split) s = g_tune_max_split;
   return s < 1 ? 1 : s;
 }
@@ -518,7 +522,7 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   P.kblocks = K_in / BK;
   // stream-K (split == 0): needs a single token tile and 128-row-aligned matrices, so that a
   // column's tile (and with it the number of partial sums to add) follows from the column index
-  bool sk = split == 0 && ztiles == 1 && max_slots >= 2 && out != nullptr;
+  bool sk = split == 0 && ztiles == 1 && max_slots >= 2 && out != nullptr && !g_tune_no_streamk;
   for (int i = 0; i < m.n && sk; ++i) sk = (m.n_out[i] % BM) == 0;
   // stream-K pays off where the per-tile decomposition cannot be split further and leaves the SMs
   // unevenly loaded (more tiles than SMs, not a whole number of two-per-SM waves); elsewhere
