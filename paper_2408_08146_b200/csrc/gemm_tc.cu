@@ -172,6 +172,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   }
   const int n_units = (int)(u_hi - u_lo);
 
+  // weight tensor map and first row of a tile
+  auto tile_map = [&](int tile, int &row0) -> const CUtensorMap * {
+    if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * BM; return &tmW2; }
+    if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * BM; return &tmW1; }
+    row0 = tile * BM;
+    return &tmW0;
+  };
+  const int pre = n_units < P.stages ? n_units : P.stages;
+
+  pdl_launch_dependents();
   if (threadIdx.x == 0) {
     for (int s = 0; s < P.stages; ++s) {
       mbar_init(&full_bar[s], 1);
@@ -184,6 +194,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     s_error = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // The weight stream starts right here, before the block-wide set-up barrier and before the
+    // dependency wait: weights do not depend on the kernel before this one.  A few more of this
+    // CTA's weight tiles are requested into L2 (bounded, so that all CTAs together stay well
+    // inside the L2).
+    int tile = (int)(u_lo / KB), kb = (int)(u_lo % KB), row0;
+    const CUtensorMap *tmW = tile_map(tile, row0);
+    const int ahead = n_units < pre + L2_AHEAD ? n_units : pre + L2_AHEAD;
+    for (int it = 0; it < ahead; ++it) {
+      if (it < pre) {
+        mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
+        tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, kb * BK, row0);
+      } else {
+        asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+                     ::"l"(tmW), "r"(kb * BK), "r"(row0) : "memory");
+      }
+      if (++kb == KB) { kb = 0; ++tile; tmW = tile_map(tile, row0); }
+    }
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
+    if (P.pair) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmXlo) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -195,40 +224,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = tmem_base_slot;
-  pdl_launch_dependents();
-
-  // weight tensor map and first row of a tile
-  auto tile_map = [&](int tile, int &row0) -> const CUtensorMap * {
-    if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * BM; return &tmW2; }
-    if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * BM; return &tmW1; }
-    row0 = tile * BM;
-    return &tmW0;
-  };
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      // (tile, K-block) of the next unit, advanced incrementally
-      int tile = (int)(u_lo / KB), kb = (int)(u_lo % KB), row0;
-      const CUtensorMap *tmW = tile_map(tile, row0);
-      asm volatile("prefetch.tensormap [%0];" ::"l"(tmW) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
-      if (P.pair) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmXlo) : "memory");
-      const int pre = n_units < P.stages ? n_units : P.stages;
-      const int ahead = n_units < pre + L2_AHEAD ? n_units : pre + L2_AHEAD;
-      // weights first: they do not depend on the kernel before this one; a few more of this CTA's
-      // weight tiles are requested into L2 while the producer of X runs (bounded, so that all CTAs
-      // together stay well inside the L2)
-      for (int it = 0; it < ahead; ++it) {
-        if (it < pre) {
-          mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
-          tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, kb * BK, row0);
-        } else {
-          asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
-                       ::"l"(tmW), "r"(kb * BK), "r"(row0) : "memory");
-        }
-        if (++kb == KB) { kb = 0; ++tile; tmW = tile_map(tile, row0); }
-      }
+      int tile, kb, row0;
+      const CUtensorMap *tmW;
       pdl_wait();
       const int lo_off = P.tt * BK * 2;          // the lo rows follow the hi rows of the tile
       tile = (int)(u_lo / KB);
