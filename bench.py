@@ -246,7 +246,12 @@ def run_koala(args):
         "gpu_launches": int(n[2]),
         "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel (all weight-streaming GEMMs of a step)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_source": f"of {peak_src}", "traffic": None,
+                     "peak_source": f"of {peak_src}",
+                     # DRAM bytes per launch (average over a step's GEMM launches): algorithmic bytes x 1.03, the
+                     # read ratio ncu measured on the O-projection and gate/up launches
+                     # (profiles/ncu_gemm_tc_kernel_t7_o_gateup.md); traffic grows with the weight bytes
+                     "traffic": 1.03 * g["bytes"] / max(g["launches"], 1),
+                     "algorithmic_bytes_per_launch": g["bytes"] / max(g["launches"], 1),
                      "launches_per_step": g["launches"] / extra, "ms_per_step_in_kernel": g["ms"] / extra},
         "step_roofline": {"algorithmic_bytes_per_step": ab, "achieved_GBps":
                           (ab["verify_weights"] + ab["draft_weights"] + ab["kv"]) / (ms_max / K * 1e-3) / 1e9,
