@@ -61,6 +61,21 @@ struct SplitIn {
   }
 };
 
+// Deferred RMSNorm scale of a GEMM input: the producer wrote x * gain (not normalised) and, per
+// row, `n` partial sums of squares; the consumer of the GEMM's output multiplies by
+// rsqrt(sum / H + eps).  n == 0: nothing pending (the input was already normalised).
+struct RowScale {
+  const float *sumsq;   // [rows][n]
+  int n;
+  float inv_h, eps;
+  __device__ __forceinline__ float of(int r) const {
+    if (n == 0) return 1.f;
+    float s = 0.f;
+    for (int i = 0; i < n; ++i) s += sumsq[(size_t)r * n + i];
+    return rsqrtf(s * inv_h + eps);
+  }
+};
+
 // Per-row plan of one forward over R rows (rows_per_seq consecutive rows per sequence).
 struct RowPlan {
   const int32_t *pos;     // [R] RoPE position
@@ -120,10 +135,14 @@ cudaError_t row_epilogue(Launch L, int dtype, int mode, float *x, SplitIn P, con
                          const void *g, Operand xn, float *out_f32, int R, int H, float eps);
 cudaError_t eagle_concat(Launch L, int dtype, const float *feat_src, const int32_t *row_src,
                          const int32_t *row_tok, const void *E, Operand cat, int R, int H, int V);
-cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowPlan plan, float *q_out,
+// x <- x + sum(P); xg <- T(x * g) (not normalised); sumsq[r][chunk] <- partial sums of x^2 over
+// chunks of 1024 columns (chunks = ceil(H / 1024)).  H % 4 == 0.
+cudaError_t row_update(Launch L, int dtype, float *x, SplitIn P, const void *g, Operand xg, float *sumsq,
+                       int R, int H);
+cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowScale sc, RowPlan plan, float *q_out,
                           void *k_cache, void *v_cache, int R, int rows_per_seq, int n_heads,
                           int head_dim, int S_max);
-cudaError_t swiglu(Launch L, int dtype, SplitIn gu, Operand act, int R, int F);
+cudaError_t swiglu(Launch L, int dtype, SplitIn gu, RowScale sc, Operand act, int R, int F);
 cudaError_t tree_attention(Launch L, int dtype, const float *q, const void *k_cache,
                            const void *v_cache, RowPlan plan, Operand out, int R, int rows_per_seq,
                            int B, int n_heads, int head_dim, int S_max);

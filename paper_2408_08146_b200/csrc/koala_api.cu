@@ -57,6 +57,8 @@ struct koala_ctx {
   size_t pcols;           // widest GEMM output
   // workspace
   float *attn_part;
+  float *sumsq[2];        // per-row partial sums of squares of the two deferred RMSNorms of a layer
+  RowScale pending;       // scale still owed by the consumer of the GEMM that reads c->xn
   int attn_chunks;
   float *x, *qbuf, *P, *verify_logits, *draft_logits, *verify_hid, *feat[2], *mx;
   Operand xn, attn_out, act, cat, lmin;
@@ -172,6 +174,8 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
   c->attn_part = (cfg.dtype == KOALA_BF16 && cfg.head_dim == 128)
                      ? w.take<float>(attn_mma_scratch_floats(Mp, cfg.n_heads, c->attn_chunks))
                      : nullptr;
+  c->sumsq[0] = w.take<float>((size_t)Mp * 8);
+  c->sumsq[1] = w.take<float>((size_t)Mp * 8);
   c->verify_tgt = w.take<int32_t>(Mp);
   c->s_parent = w.take<int32_t>(N);
   c->s_level = w.take<int32_t>(N);
@@ -277,15 +281,23 @@ int do_gemm(koala_ctx *c, Operand X, int K_in, GemmMats m, int R, float *direct,
 // One pre-norm decoder layer over R rows.  On entry x holds the residual stream and xn the
 // normalised input of the attention block.  On exit x is updated and `next_xn` holds
 // T(rmsnorm(x) * next_g) (or T(x) if next_g is null); `out_f32` optionally receives the same in fp32.
+// One pre-norm decoder layer over R rows.  On entry x holds the residual stream and xn the input
+// of the attention block: normalised, or x * gain with the scale still pending in c->pending.
+// On exit x is updated; if `defer` the next layer's input is left in c->xn as x * next_g with its
+// scale pending, otherwise `next_xn` holds T(rmsnorm(x) * next_g) (or T(x) if next_g is null) and
+// `out_f32` optionally the same in fp32.
 int run_layer(koala_ctx *c, const LayerW &w, void *kc, void *vc, int R, int rows_per_seq,
-              const void *next_g, Operand next_xn, float *out_f32) {
+              const void *next_g, Operand next_xn, float *out_f32, bool defer) {
   const koala_config &g = c->cfg;
   const int H = g.H, F = g.F;
+  const bool can_defer = (H % 4) == 0 && H <= 8192;
+  const RowScale none{nullptr, 0, 0.f, 0.f};
   SplitIn s;
   GemmMats qkv{{w.wq, w.wk, w.wv}, {H, H, H}, 3};
   K_TRY(do_gemm(c, c->xn, H, qkv, R, nullptr, 0, &s));
-  CU_TRY(rope_kv_write(LN(c), g.dtype, s, row_plan(c), c->qbuf, kc, vc, R, rows_per_seq, g.n_heads,
+  CU_TRY(rope_kv_write(LN(c), g.dtype, s, c->pending, row_plan(c), c->qbuf, kc, vc, R, rows_per_seq, g.n_heads,
                        g.head_dim, g.S_max));
+  c->pending = none;
   const int ta = time_begin(c, KOALA_CLS_ATTENTION, 0);
   if (c->use_tc && g.head_dim == 128 && c->attn_part != nullptr && rows_per_seq <= 128) {
     CU_TRY(tree_attention_mma(LN(c), c->qbuf, kc, vc, row_plan(c), c->attn_out, c->attn_part, rows_per_seq,
@@ -298,13 +310,24 @@ int run_layer(koala_ctx *c, const LayerW &w, void *kc, void *vc, int R, int rows
   time_end(c, ta);
   GemmMats o{{w.wo, nullptr, nullptr}, {H, 0, 0}, 1};
   K_TRY(do_gemm(c, c->attn_out, H, o, R, nullptr, 0, &s));
-  CU_TRY(row_epilogue(LN(c), g.dtype, 0, c->x, s, nullptr, w.ffn_norm, c->xn, nullptr, R, H, g.rms_eps));
+  RowScale ffn = none;
+  if (can_defer && (s.ld % 4) == 0 && (s.stride % 4) == 0) {
+    CU_TRY(row_update(LN(c), g.dtype, c->x, s, w.ffn_norm, c->xn, c->sumsq[0], R, H));
+    ffn = RowScale{c->sumsq[0], (H + 1023) / 1024, 1.f / (float)H, g.rms_eps};
+  } else {
+    CU_TRY(row_epilogue(LN(c), g.dtype, 0, c->x, s, nullptr, w.ffn_norm, c->xn, nullptr, R, H, g.rms_eps));
+  }
   GemmMats gu{{w.wg, w.wu, nullptr}, {F, F, 0}, 2};
   K_TRY(do_gemm(c, c->xn, H, gu, R, nullptr, 0, &s));
-  CU_TRY(swiglu(LN(c), g.dtype, s, c->act, R, F));
+  CU_TRY(swiglu(LN(c), g.dtype, s, ffn, c->act, R, F));
   GemmMats dn{{w.wd, nullptr, nullptr}, {H, 0, 0}, 1};
   K_TRY(do_gemm(c, c->act, F, dn, R, nullptr, 0, &s));
-  CU_TRY(row_epilogue(LN(c), g.dtype, 0, c->x, s, nullptr, next_g, next_xn, out_f32, R, H, g.rms_eps));
+  if (defer && can_defer && next_g != nullptr && (s.ld % 4) == 0 && (s.stride % 4) == 0) {
+    CU_TRY(row_update(LN(c), g.dtype, c->x, s, next_g, c->xn, c->sumsq[1], R, H));
+    c->pending = RowScale{c->sumsq[1], (H + 1023) / 1024, 1.f / (float)H, g.rms_eps};
+  } else {
+    CU_TRY(row_epilogue(LN(c), g.dtype, 0, c->x, s, nullptr, next_g, next_xn, out_f32, R, H, g.rms_eps));
+  }
   return KOALA_OK;
 }
 
@@ -317,6 +340,7 @@ int draft_eagle(koala_ctx *c, int pass) {
   const int H = g.H, k = g.topk, B = g.B;
   const int rows = pass == 0 ? c->pend_cap : k;
   const int R = B * rows;
+  c->pending = RowScale{nullptr, 0, 0.f, 0.f};
   const float *feat_src;
   if (pass == 0) {
     CU_TRY(plan_draft0(LN(c), c->t, c->p, c->seq_len, B, g.N, rows, g.head_dim, g.rope_base, g.S_max,
@@ -346,7 +370,7 @@ int draft_eagle(koala_ctx *c, int pass) {
       const bool last = j == g.K - 1;
       K_TRY(run_layer(c, c->draft_layers[j], (unsigned char *)c->dk + j * le, (unsigned char *)c->dv + j * le,
                       R, rows, last ? nullptr : c->draft_layers[j + 1].attn_norm, last ? lm_all : c->xn,
-                      last ? f_all : nullptr));
+                      last ? f_all : nullptr, !last));
     }
   }
   int lm_rows = R;
@@ -487,6 +511,7 @@ int koala_init(const koala_config *cfg, const koala_weights *w, const koala_stat
   c->pend_cap = g.N < g.D + 1 ? g.N : g.D + 1;
   c->draft_rows = 0;
   c->expand_mode = 0;
+  c->pending = RowScale{nullptr, 0, 0.f, 0.f};
   c->timing = false;
   c->ev_used = 0;
   memset(c->t_bytes, 0, sizeof(c->t_bytes));
@@ -551,6 +576,7 @@ int koala_verify(koala_ctx *c, const koala_tree *tree) {
     c->pend_cap = g.N < g.D + 1 ? g.N : g.D + 1;
   }
   const int R = g.B * g.N;
+  c->pending = RowScale{nullptr, 0, 0.f, 0.f};
   CU_TRY(tree_ancestors(LN(c), c->t, g.B, g.N));
   CU_TRY(plan_verify(LN(c), c->t, c->p, c->seq_len, g.B, g.N, g.head_dim, g.rope_base, g.S_max, c->status));
   CU_TRY(embed_norm(LN(c), g.dtype, c->p.row_tok, c->embed, c->layers[0].attn_norm, c->x, c->xn, R, g.H, g.V,
@@ -560,7 +586,7 @@ int koala_verify(koala_ctx *c, const koala_tree *tree) {
     const bool last = l == g.L - 1;
     K_TRY(run_layer(c, c->layers[l], (unsigned char *)c->tk + l * le, (unsigned char *)c->tv + l * le, R, g.N,
                     last ? c->final_norm : c->layers[l + 1].attn_norm, last ? c->lmin : c->xn,
-                    last ? c->verify_hid : nullptr));
+                    last ? c->verify_hid : nullptr, !last));
   }
   GemmMats lm{{c->lm_head, nullptr, nullptr}, {g.V, 0, 0}, 1};
   K_TRY(do_gemm(c, c->lmin, g.H, lm, R, c->verify_logits, g.V, nullptr));

@@ -189,6 +189,33 @@ row_epilogue_vec_kernel(int mode, float *__restrict__ x, SplitIn P, const T *__r
   }
 }
 
+// Residual update with the RMSNorm deferred: grid (chunks of 1024 columns, rows).  Many CTAs per
+// row pull the split-K partial sums; the row statistic is left as per-chunk partial sums of
+// squares for the consumer of the next GEMM's output (RowScale).
+template <typename T>
+__global__ void __launch_bounds__(256)
+row_update_kernel(float *__restrict__ x, SplitIn P, const T *__restrict__ g, T *__restrict__ xg,
+                  T *__restrict__ xg_lo, float *__restrict__ sumsq, int H) {
+  __shared__ float red[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.y;
+  const int c = (blockIdx.x * 256 + threadIdx.x) * 4;
+  float ss = 0.f;
+  if (c < H) {
+    const float4 gg = load4<T>(g + c);
+    const float4 p = split_sum4(P, r, c);
+    float *xr = x + (size_t)r * H + c;
+    const float4 xv = *reinterpret_cast<const float4 *>(xr);
+    const float4 o = make_float4(xv.x + p.x, xv.y + p.y, xv.z + p.z, xv.w + p.w);
+    *reinterpret_cast<float4 *>(xr) = o;
+    ss = o.x * o.x + o.y * o.y + o.z * o.z + o.w * o.w;
+    store_operand4(xg, xg_lo, (size_t)r * H + c, make_float4(o.x * gg.x, o.y * gg.y, o.z * gg.z, o.w * gg.w));
+  }
+  const float tot = block_sum(ss, red);
+  if (threadIdx.x == 0) sumsq[(size_t)r * gridDim.x + blockIdx.x] = tot;
+}
+
 // ------------------------------------------------------------------------------- EAGLE fc input
 template <typename T>
 __global__ void eagle_concat_kernel(const float *__restrict__ feat_src,
@@ -237,7 +264,7 @@ __global__ void reduce_splits_kernel(SplitIn P, float *__restrict__ Y, int ldy, 
 // ------------------------------------------------------------------------------- RoPE + KV write
 // grid (R, n_heads), block head_dim/2: thread i rotates the pair (i, i + head_dim/2).
 template <typename T>
-__global__ void rope_kv_kernel(SplitIn qkv, RowPlan plan, float *__restrict__ q_out,
+__global__ void rope_kv_kernel(SplitIn qkv, RowScale sc, RowPlan plan, float *__restrict__ q_out,
                                T *__restrict__ k_cache, T *__restrict__ v_cache, int rows_per_seq,
                                int n_heads, int head_dim, int S_max) {
   pdl_launch_dependents();
@@ -248,12 +275,13 @@ __global__ void rope_kv_kernel(SplitIn qkv, RowPlan plan, float *__restrict__ q_
   const int slot = plan.slot[r];
   const float2 cs = plan.rope[(size_t)r * half + i];
   const int c0 = h * head_dim + i, c1 = c0 + half;
-  const float q0 = qkv.at(r, c0), q1 = qkv.at(r, c1);
+  const float rs = sc.of(r);
+  const float q0 = rs * qkv.at(r, c0), q1 = rs * qkv.at(r, c1);
   q_out[(size_t)r * H + c0] = q0 * cs.x - q1 * cs.y;
   q_out[(size_t)r * H + c1] = q1 * cs.x + q0 * cs.y;
   if (slot < 0 || slot >= S_max) return;
-  const float k0 = qkv.at(r, H + c0), k1 = qkv.at(r, H + c1);
-  const float v0 = qkv.at(r, 2 * H + c0), v1 = qkv.at(r, 2 * H + c1);
+  const float k0 = rs * qkv.at(r, H + c0), k1 = rs * qkv.at(r, H + c1);
+  const float v0 = rs * qkv.at(r, 2 * H + c0), v1 = rs * qkv.at(r, 2 * H + c1);
   const size_t base = (((size_t)b * n_heads + h) * S_max + slot) * head_dim;
   k_cache[base + i] = from_f<T>(k0 * cs.x - k1 * cs.y);
   k_cache[base + i + half] = from_f<T>(k1 * cs.x + k0 * cs.y);
@@ -279,7 +307,7 @@ __device__ __forceinline__ void store2(bf16 *p, float a, float b) {
 }
 template <typename T>
 __global__ void __launch_bounds__(1024)
-rope_kv_vec_kernel(SplitIn qkv, RowPlan plan, float *__restrict__ q_out, T *__restrict__ k_cache,
+rope_kv_vec_kernel(SplitIn qkv, RowScale sc, RowPlan plan, float *__restrict__ q_out, T *__restrict__ k_cache,
                    T *__restrict__ v_cache, int rows_per_seq, int n_heads, int head_dim, int S_max) {
   pdl_launch_dependents();
   pdl_wait();
@@ -288,16 +316,21 @@ rope_kv_vec_kernel(SplitIn qkv, RowPlan plan, float *__restrict__ q_out, T *__re
   const int b = r / rows_per_seq;
   const int slot = plan.slot[r];
   const bool wr = slot >= 0 && slot < S_max;
-  for (int p = threadIdx.x; p < n_heads * hq; p += blockDim.x) {
+  const float rs = sc.of(r);
+  // grid.y slices the row's work so that many SMs pull the partial sums
+  for (int p = blockIdx.y * blockDim.x + threadIdx.x; p < n_heads * hq; p += gridDim.y * blockDim.x) {
     const int h = p / hq, i = (p - h * hq) * 2;
     const float4 cs = *reinterpret_cast<const float4 *>(&plan.rope[(size_t)r * half + i]);   // c0 s0 c1 s1
     const int c0 = h * head_dim + i, c1 = c0 + half;
-    const float2 qa = split_sum2(qkv, r, c0), qb = split_sum2(qkv, r, c1);
+    float2 qa = split_sum2(qkv, r, c0), qb = split_sum2(qkv, r, c1);
+    qa.x *= rs; qa.y *= rs; qb.x *= rs; qb.y *= rs;
     store2(q_out + (size_t)r * H + c0, qa.x * cs.x - qb.x * cs.y, qa.y * cs.z - qb.y * cs.w);
     store2(q_out + (size_t)r * H + c1, qb.x * cs.x + qa.x * cs.y, qb.y * cs.z + qa.y * cs.w);
     if (!wr) continue;
-    const float2 ka = split_sum2(qkv, r, H + c0), kb = split_sum2(qkv, r, H + c1);
-    const float2 va = split_sum2(qkv, r, 2 * H + c0), vb = split_sum2(qkv, r, 2 * H + c1);
+    float2 ka = split_sum2(qkv, r, H + c0), kb = split_sum2(qkv, r, H + c1);
+    float2 va = split_sum2(qkv, r, 2 * H + c0), vb = split_sum2(qkv, r, 2 * H + c1);
+    ka.x *= rs; ka.y *= rs; kb.x *= rs; kb.y *= rs;
+    va.x *= rs; va.y *= rs; vb.x *= rs; vb.y *= rs;
     const size_t base = (((size_t)b * n_heads + h) * S_max + slot) * head_dim + i;
     store2(k_cache + base, ka.x * cs.x - kb.x * cs.y, ka.y * cs.z - kb.y * cs.w);
     store2(k_cache + base + half, kb.x * cs.x + ka.x * cs.y, kb.y * cs.z + ka.y * cs.w);
@@ -308,25 +341,28 @@ rope_kv_vec_kernel(SplitIn qkv, RowPlan plan, float *__restrict__ q_out, T *__re
 
 // ------------------------------------------------------------------------------- SwiGLU
 template <typename T>
-__global__ void swiglu_kernel(SplitIn gu, T *__restrict__ act, T *__restrict__ act_lo, int F) {
+__global__ void swiglu_kernel(SplitIn gu, RowScale sc, T *__restrict__ act, T *__restrict__ act_lo, int F) {
   pdl_launch_dependents();
   pdl_wait();
   const int r = blockIdx.y;
   const int f = blockIdx.x * blockDim.x + threadIdx.x;
   if (f >= F) return;
-  store_operand(act, act_lo, (size_t)r * F + f, silu_f(gu.at(r, f)) * gu.at(r, F + f));
+  const float rs = sc.of(r);
+  store_operand(act, act_lo, (size_t)r * F + f, silu_f(rs * gu.at(r, f)) * (rs * gu.at(r, F + f)));
 }
 
 template <typename T>
-__global__ void swiglu_vec_kernel(SplitIn gu, T *__restrict__ act, T *__restrict__ act_lo, int F) {
+__global__ void swiglu_vec_kernel(SplitIn gu, RowScale sc, T *__restrict__ act, T *__restrict__ act_lo, int F) {
   pdl_launch_dependents();
   pdl_wait();
   const int r = blockIdx.y;
   const int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (f >= F) return;
+  const float rs = sc.of(r);
   const float4 a = split_sum4(gu, r, f), b = split_sum4(gu, r, F + f);
   store_operand4(act, act_lo, (size_t)r * F + f,
-                 make_float4(silu_f(a.x) * b.x, silu_f(a.y) * b.y, silu_f(a.z) * b.z, silu_f(a.w) * b.w));
+                 make_float4(silu_f(rs * a.x) * (rs * b.x), silu_f(rs * a.y) * (rs * b.y),
+                             silu_f(rs * a.z) * (rs * b.z), silu_f(rs * a.w) * (rs * b.w)));
 }
 
 // ------------------------------------------------------------------------------- tree attention
@@ -538,28 +574,36 @@ cudaError_t reduce_splits(Launch L, SplitIn P, float *Y, int ldy, int R, int nco
                   ldy, ncols);
 }
 
-cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowPlan plan, float *q_out,
+cudaError_t row_update(Launch L, int dtype, float *x, SplitIn P, const void *g, Operand xg, float *sumsq,
+                       int R, int H) {
+  if (H % 4 != 0 || P.ld % 4 != 0 || P.stride % 4 != 0) return cudaErrorInvalidValue;
+  DISPATCH_T(dtype, return launch_k(row_update_kernel<T>, dim3((H + 1023) / 1024, R), dim3(256), 0, L.st, L.pdl,
+                                    x, P, (const T *)g, (T *)xg.hi, (T *)xg.lo, sumsq, H);)
+}
+
+cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowScale sc, RowPlan plan, float *q_out,
                           void *k_cache, void *v_cache, int R, int rows_per_seq, int n_heads,
                           int head_dim, int S_max) {
   if (head_dim % 4 == 0 && qkv.ld % 2 == 0 && qkv.stride % 2 == 0) {
     const int work = n_heads * head_dim / 4;
-    const int threads = work < 1024 ? ((work + 31) / 32) * 32 : 1024;
-    DISPATCH_T(dtype, return launch_k(rope_kv_vec_kernel<T>, dim3(R), dim3(threads), 0, L.st, L.pdl, qkv, plan,
+    const int threads = work < 128 ? ((work + 31) / 32) * 32 : 128;
+    const int slices = (work + threads - 1) / threads;
+    DISPATCH_T(dtype, return launch_k(rope_kv_vec_kernel<T>, dim3(R, slices), dim3(threads), 0, L.st, L.pdl, qkv, sc, plan,
                                       q_out, (T *)k_cache, (T *)v_cache, rows_per_seq, n_heads, head_dim,
                                       S_max);)
   }
   DISPATCH_T(dtype, return launch_k(rope_kv_kernel<T>, dim3(R, n_heads), dim3(head_dim / 2), 0, L.st,
-                                    L.pdl, qkv, plan, q_out, (T *)k_cache, (T *)v_cache,
+                                    L.pdl, qkv, sc, plan, q_out, (T *)k_cache, (T *)v_cache,
                                     rows_per_seq, n_heads, head_dim, S_max);)
 }
 
-cudaError_t swiglu(Launch L, int dtype, SplitIn gu, Operand act, int R, int F) {
+cudaError_t swiglu(Launch L, int dtype, SplitIn gu, RowScale sc, Operand act, int R, int F) {
   if (F % 4 == 0 && gu.ld % 4 == 0 && gu.stride % 4 == 0) {
     DISPATCH_T(dtype, return launch_k(swiglu_vec_kernel<T>, dim3((F / 4 + 255) / 256, R), dim3(256), 0, L.st,
-                                      L.pdl, gu, (T *)act.hi, (T *)act.lo, F);)
+                                      L.pdl, gu, sc, (T *)act.hi, (T *)act.lo, F);)
   }
   DISPATCH_T(dtype, return launch_k(swiglu_kernel<T>, dim3((F + 255) / 256, R), dim3(256), 0, L.st,
-                                    L.pdl, gu, (T *)act.hi, (T *)act.lo, F);)
+                                    L.pdl, gu, sc, (T *)act.hi, (T *)act.lo, F);)
 }
 
 cudaError_t tree_attention(Launch L, int dtype, const float *q, const void *k_cache,
