@@ -265,11 +265,50 @@ def run_koala(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_oracle_leg(cfg, store, steps=1, warmup=1)
     eng.close()
+    del eng
+    if rank == 0 and world == 1:
+        line["autoregressive"] = autoregressive_leg(cfg, store, dev, steps=max(K, 8))
+        line["autoregressive"]["speedup_ratio_at_forced_acceptance"] = line["value"] / line["autoregressive"]["value"]
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def autoregressive_leg(cfg, store, dev, steps: int):
+    """Vanilla autoregressive decoding with the same target (the denominator of the paper's wall-time
+    speed-up ratio, Section 4.1): every step verifies a one-node tree and accepts its bonus token."""
+    from paper_2408_08146_b200 import Koala
+    ar_cfg = cfg.with_(name=cfg.name + "_ar", N=1, S_max=cfg.prompt_len + steps + 80)
+    one = np.asarray([-1], np.int32), np.asarray([0], np.int32), np.asarray([0], np.int32)
+    eng = Koala(ar_cfg, store.tensors, static_tree=one, device=dev)
+    pr = prompts(cfg)
+    # one-node chains: the prompt is ingested token by token here, so seed the cache length instead
+    eng.seq_len.fill_(cfg.prompt_len)
+    bufs = eng.buffers()
+    par = torch.full((cfg.B, 1), -1, dtype=torch.int32, device=dev)
+    n1 = torch.ones(cfg.B, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        eng.koala_verify((bufs["root_tok"].view(cfg.B, 1), par, n1, 1))
+        eng.koala_accept(None)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert eng.device_status() == 0
+    eng.close()
+    return {"value": cfg.B / (ms * 1e-3), "unit": UNIT, "ms_per_token": ms, "steps": steps,
+            "note": "same target, one-node tree per step, cache length seeded at the prompt length"}
 
 
 # ------------------------------------------------------------------------------------------------
