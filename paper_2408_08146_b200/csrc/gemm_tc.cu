@@ -39,7 +39,8 @@ constexpr int W_STAGE_BYTES = BM * BK * 2;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // about a second of SM clock
 constexpr int E_TIMEOUT = 6;
 constexpr int MAX_STAGES = 12;
-constexpr int L2_AHEAD = 8;          // weight tiles (16 KB each) prefetched into L2 beyond the ring
+constexpr int L2_AHEAD = 0;          // weight tiles (16 KB each) prefetched into L2 beyond the ring (measured: any
+                                     // depth slows the small kernels that run meanwhile more than it helps)
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -131,6 +132,8 @@ struct TcParams {
   unsigned sk_units;  // tiles * kblocks
   size_t split_stride;
   int stages;
+  int early_w;        // 1: the first stages' weight tiles are requested before the dependency wait
+  int l2_ahead;       // weight tiles prefetched into L2 beyond the ring before the dependency wait
   int *status;
 };
 
@@ -200,7 +203,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     // inside the L2).
     int tile = (int)(u_lo / KB), kb = (int)(u_lo % KB), row0;
     const CUtensorMap *tmW = tile_map(tile, row0);
-    const int ahead = n_units < pre + L2_AHEAD ? n_units : pre + L2_AHEAD;
+    const int ahead = P.early_w ? (n_units < pre + P.l2_ahead ? n_units : pre + P.l2_ahead) : 0;
     for (int it = 0; it < ahead; ++it) {
       if (it < pre) {
         mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
@@ -237,6 +240,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       tmW = tile_map(tile, row0);
       for (int it = 0; it < pre; ++it) {
         unsigned char *xd = tiles + (size_t)it * stage_bytes + W_STAGE_BYTES;
+        if (!P.early_w) {
+          mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
+          tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, kb * BK, row0);
+        }
         tma_load_2d(&tmX, &full_bar[it], xd, kb * BK, tok0);
         if (P.pair) tma_load_2d(&tmXlo, &full_bar[it], xd + lo_off, kb * BK, tok0);
         if (++kb == KB) { kb = 0; ++tile; tmW = tile_map(tile, row0); }
@@ -378,6 +385,8 @@ int g_num_sms = 148;
 int g_tune_stages = 0;      // 0 = as many as fit (at most 8)
 int g_tune_max_split = 0;   // 0 = default rule
 int g_tune_no_streamk = 0;  // 1 = always the per-tile decomposition
+int g_tune_l2_ahead = -1;   // < 0 = default
+int g_tune_late_w = 0;      // 1 = weights wait for the dependency too
 
 bool get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out) {
   std::lock_guard<std::mutex> lock(g_mu);
@@ -431,6 +440,8 @@ void tc_set_tuning(int key, int value) {
   if (key == 1) g_tune_stages = value;
   if (key == 2) g_tune_max_split = value;
   if (key == 3) g_tune_no_streamk = value;
+  if (key == 5) g_tune_l2_ahead = value;
+  if (key == 6) g_tune_late_w = value;
 }
 
 void tc_forget_maps() {
@@ -560,6 +571,8 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   if (g_tune_stages > 0 && g_tune_stages < stages) stages = g_tune_stages;
   if (stages < 2) return cudaErrorInvalidValue;
   P.stages = stages;
+  P.l2_ahead = g_tune_l2_ahead >= 0 ? g_tune_l2_ahead : L2_AHEAD;
+  P.early_w = g_tune_late_w ? 0 : 1;
   CUtensorMap mw[3], mx, mxlo;
   for (int i = 0; i < 3; ++i) {
     const int j = i < m.n ? i : 0;
