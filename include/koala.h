@@ -213,7 +213,9 @@ int koala_timing_read(koala_ctx *ctx, koala_timing *out);
 /* Process-wide tuning of the tensor-core matrix multiply (for sweeps; the defaults are chosen
  * for B200): key 1 = shared-memory pipeline stages per CTA (0 = as many as fit, at most 8);
  * key 2 = upper bound on the automatic split-K factor (0 = default); key 3 = 1 switches stream-K
- * off (every CTA stays inside one weight tile). */
+ * off (every CTA stays inside one weight tile); key 5 = weight tiles prefetched into L2 ahead of the
+ * pipeline (< 0 = default 0); key 6 = 1 delays the weight stream until the previous kernel has
+ * finished; key 7 = divisor of the split-K partial-sum traffic bound (default 8). */
 void koala_set_tuning(int key, int value);
 
 /* Kernels launched by the library in this process so far (all contexts). */

@@ -387,6 +387,7 @@ int g_tune_max_split = 0;   // 0 = default rule
 int g_tune_no_streamk = 0;  // 1 = always the per-tile decomposition
 int g_tune_l2_ahead = -1;   // < 0 = default
 int g_tune_late_w = 0;      // 1 = weights wait for the dependency too
+int g_tune_traffic_div = 8; // split <= K_in / (div * tokens)
 
 bool get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out) {
   std::lock_guard<std::mutex> lock(g_mu);
@@ -442,6 +443,7 @@ void tc_set_tuning(int key, int value) {
   if (key == 3) g_tune_no_streamk = value;
   if (key == 5) g_tune_l2_ahead = value;
   if (key == 6) g_tune_late_w = value;
+  if (key == 7 && value > 0) g_tune_traffic_div = value;
 }
 
 void tc_forget_maps() {
@@ -463,7 +465,7 @@ int tc_default_split(int n_tiles, int kblocks, int tokens) {
   const int slots = 2 * g_num_sms;
   int s = slots / (n_tiles > 0 ? n_tiles : 1);
   const int by_k = kblocks / 8;
-  const int by_traffic = (kblocks * 64) / (8 * (tokens > 0 ? tokens : 1));
+  const int by_traffic = (kblocks * 64) / (g_tune_traffic_div * (tokens > 0 ? tokens : 1));
   if (s > by_k) s = by_k;
   if (s > by_traffic) s = by_traffic;
   if (s > 8) s = 8;
@@ -481,7 +483,7 @@ int tc_streamk_ctas(int n_tiles, int kblocks, int tokens, int max_slots, int *sl
   if (g > units / 8) g = units / 8;
   if (g < 1) g = 1;
   // average contributors per tile = kblocks * g / units; bound it by the traffic rule
-  const long long by_traffic = (long long)(kblocks * 64) / (8LL * (tokens > 0 ? tokens : 1));
+  const long long by_traffic = (long long)(kblocks * 64) / ((long long)g_tune_traffic_div * (tokens > 0 ? tokens : 1));
   const long long avg_cap = by_traffic < 1 ? 1 : by_traffic;
   if ((long long)kblocks * g > avg_cap * units) g = avg_cap * units / kblocks;
   if (g_tune_max_split > 0 && (long long)kblocks * g > (long long)g_tune_max_split * units)
