@@ -1,0 +1,156 @@
+"""Edge cases of the CUDA path against the oracle: degenerate trees, maximum tree size, a head
+without layers, long contexts that span many key tiles and several key chunks, capacity and
+malformed-input reporting, and the call-order rules."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from oracle.koala_oracle import KoalaOracle, round_to_bf16
+from paper_2408_08146_b200 import Koala, KoalaError
+from tests.harness import kv_to_oracle, make_pair, tok_list
+from tests.parity import assert_close, check_argmax
+from workloads import T7_EAGLE, TINY_EAGLE, reduced
+from workloads.generate import prompts, random_kv, uniform_ints
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _tree_arrays(eng, toks, parents):
+    cfg = eng.cfg
+    n = len(toks[0])
+    to = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(DEV)
+    return to(toks), to(parents), to(np.full(cfg.B, n)), n
+
+
+def test_single_node_tree_is_plain_autoregressive_decoding():
+    cfg = TINY_EAGLE.with_(N=1, D=1, S_max=128)
+    eng, orc, _ = make_pair(cfg)
+    pr = prompts(cfg)
+    # one token per call: 64 single-node chains, forced acceptance of 1 = the node itself
+    for t in range(cfg.prompt_len):
+        tree = _tree_arrays(eng, [[int(pr[0][t])]], [[-1]])
+        eng.koala_verify(tree)
+        eng.koala_accept(tree[2])
+    orc.prefill(pr, 1)
+    out = []
+    for _ in range(6):
+        root = eng.buffers()["root_tok"].cpu().numpy().reshape(1, 1)
+        eng.koala_verify(_tree_arrays(eng, root, [[-1]]))
+        tk, ln = tok_list(*eng.koala_accept(None))
+        assert ln == [1]
+        out += tk[0]
+    assert out == orc.ar_greedy(6)[0]
+    assert eng.device_status() == 0
+    eng.close()
+
+
+def test_maximum_tree_of_128_nodes_chain_and_bushy():
+    cfg = TINY_EAGLE.with_(N=128, D=4, topk=2, S_max=400, prompt_len=128)
+    eng, orc, _ = make_pair(cfg)
+    pr = prompts(cfg)
+    eng.prefill(pr, 128)                     # one chain of 128 nodes: every mask bit in use
+    orc.prefill(pr, 128)
+    assert eng.seq_len.cpu().tolist() == orc.seq_len == [128]
+    for l in range(cfg.L):
+        assert_close(kv_to_oracle(eng.target_k, l, 0, np.float64)[:128], orc.target_k[l][0][:128], cfg.dtype, "K")
+    # a bushy 128-node caller tree on top of it
+    n = 128
+    par = [-1] + [int(p) for p in (uniform_ints(5, "edge.par", n - 1, 0, 1 << 20) % np.arange(1, n))]
+    par = [-1 if u == 0 else min(par[u], u - 1) for u in range(n)]
+    tok = uniform_ints(5, "edge.tok", n, 0, cfg.V)
+    tok[0] = orc.root_tok[0]
+    eng.koala_verify(_tree_arrays(eng, [tok], [par]))
+    orc.verify([(tok, np.asarray(par))])
+    b = eng.buffers()
+    assert_close(b["verify_logits"][:n].cpu().numpy(), orc.verify_logits[0], cfg.dtype, "128-node tree logits")
+    check_argmax(b["verify_tgt"][:n].cpu().numpy(), orc.verify_logits[0], "128-node tree arg-max")
+    got = tok_list(*eng.koala_accept(None))
+    ref = orc.accept()
+    assert list(got[0]) == list(ref[0]) and list(got[1]) == list(ref[1])
+    assert eng.device_status() == 0
+    eng.close()
+
+
+def test_eagle_head_without_layers():
+    cfg = TINY_EAGLE.with_(K=0, S_max=160)
+    eng, orc, _ = make_pair(cfg)
+    pr = prompts(cfg)
+    eng.prefill(pr, 15)
+    orc.prefill(pr, 15)
+    for _ in range(2):
+        got = tok_list(*eng.step())
+        ref = orc.step()
+        assert list(got[0]) == ref[0] and list(got[1]) == ref[1]
+        n = len(orc.tree_tok[0])
+        assert eng.buffers()["tree_tok"][0, :n].cpu().tolist() == list(orc.tree_tok[0])
+    assert eng.device_status() == 0
+    eng.close()
+
+
+@pytest.mark.parametrize("context", [1000, 3900])
+def test_long_context_many_key_tiles_and_chunks(context):
+    """bf16, head_dim 128, one 7B-shaped layer: the attention kernel walks dozens of key tiles and,
+    at the longer context, several key chunks merged by the second kernel."""
+    cfg = reduced(T7_EAGLE, 1, K=1, N=60, S_max=4096, prompt_len=context)
+    eng, orc, _ = make_pair(cfg, oracle_dtype=np.float32, cache_host=False)
+    eng.target_k.copy_(random_kv(cfg, "target_k", cfg.L, DEV))
+    eng.target_v.copy_(random_kv(cfg, "target_v", cfg.L, DEV))
+    orc.target_k[0][0][...] = kv_to_oracle(eng.target_k, 0, 0, np.float32)
+    orc.target_v[0][0][...] = kv_to_oracle(eng.target_v, 0, 0, np.float32)
+    eng.seq_len.fill_(context)
+    orc.seq_len[0] = context
+    n = cfg.N
+    par = [-1] + [max(0, u - 1 - (u * 7) % min(u, 5)) for u in range(1, n)]
+    tok = uniform_ints(9, "edge.long", n, 0, cfg.V)
+    eng.koala_verify(_tree_arrays(eng, [tok], [par]))
+    orc.verify([(tok, np.asarray(par))])
+    b = eng.buffers()
+    assert_close(b["verify_hid"][:n].cpu().numpy(), orc.verify_hid[0], cfg.dtype, f"hidden at context {context}")
+    assert_close(b["verify_logits"][:n].cpu().numpy(), orc.verify_logits[0], cfg.dtype, f"logits at context {context}")
+    assert eng.device_status() == 0
+    eng.close()
+
+
+def test_capacity_and_malformed_trees_are_reported_not_executed():
+    cfg = TINY_EAGLE.with_(S_max=80)                    # the 64-token prompt fits, prompt + tree does not
+    eng, orc, _ = make_pair(cfg)
+    pr = prompts(cfg)
+    eng.prefill(pr, 15)
+    assert eng.device_status() == 0
+    eng.seq_len.fill_(70)                               # 70 + 15 > 80
+    k_before = eng.target_k.clone()
+    eng.koala_verify(_tree_arrays(eng, [[1] * 15], [list(range(-1, 14))]))
+    assert eng.device_status() == 3                     # KOALA_E_CAPACITY, from the plan kernel
+    assert torch.equal(k_before, eng.target_k)          # nothing was written past the capacity
+    eng.close()
+    eng, _, _ = make_pair(TINY_EAGLE)
+    eng.koala_verify(_tree_arrays(eng, [[1, 2, 3]], [[-1, 2, 0]]))     # parent index not below the child
+    assert eng.device_status() == 1                     # KOALA_E_INVALID
+    eng.close()
+
+
+def test_call_order_and_argument_errors():
+    eng, _, _ = make_pair(TINY_EAGLE)
+    with pytest.raises(KoalaError) as e:
+        eng.koala_expand_tree(0)                        # nothing drafted
+    assert e.value.code == 4
+    with pytest.raises(KoalaError) as e:
+        eng.koala_draft(1)                              # pass 1 before pass 0
+    assert e.value.code == 4
+    with pytest.raises(KoalaError) as e:
+        eng.koala_draft(99)
+    assert e.value.code == 1
+    with pytest.raises(KoalaError) as e:
+        eng.koala_verify(None)                          # no drafted tree
+    assert e.value.code == 4
+    with pytest.raises(KoalaError) as e:
+        eng.koala_accept(None)                          # nothing verified
+    assert e.value.code == 4
+    tok = torch.zeros(1, 16, dtype=torch.int32, device=DEV)
+    with pytest.raises(KoalaError) as e:
+        eng.koala_verify((tok, tok, torch.ones(1, dtype=torch.int32, device=DEV), 16))   # n_max > N
+    assert e.value.code == 1
+    eng.close()
