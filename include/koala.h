@@ -215,7 +215,8 @@ int koala_timing_read(koala_ctx *ctx, koala_timing *out);
  * key 2 = upper bound on the automatic split-K factor (0 = default); key 3 = 1 switches stream-K
  * off (every CTA stays inside one weight tile); key 5 = weight tiles prefetched into L2 ahead of the
  * pipeline (< 0 = default 0); key 6 = 1 delays the weight stream until the previous kernel has
- * finished; key 7 = divisor of the split-K partial-sum traffic bound (default 8). */
+ * finished; key 7 = divisor of the split-K partial-sum traffic bound (default 8); key 8 = how many
+ * pipeline stages request their weight tile before that wait (< 0 = all, the default). */
 void koala_set_tuning(int key, int value);
 
 /* Kernels launched by the library in this process so far (all contexts). */

@@ -132,7 +132,7 @@ struct TcParams {
   unsigned sk_units;  // tiles * kblocks
   size_t split_stride;
   int stages;
-  int early_w;        // 1: the first stages' weight tiles are requested before the dependency wait
+  int early_w;        // how many of the first stages' weight tiles are requested before the dependency wait
   int l2_ahead;       // weight tiles prefetched into L2 beyond the ring before the dependency wait
   int *status;
 };
@@ -203,9 +203,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     // inside the L2).
     int tile = (int)(u_lo / KB), kb = (int)(u_lo % KB), row0;
     const CUtensorMap *tmW = tile_map(tile, row0);
-    const int ahead = P.early_w ? (n_units < pre + P.l2_ahead ? n_units : pre + P.l2_ahead) : 0;
+    const int early = pre < P.early_w ? pre : P.early_w;
+    const int ahead = early == pre ? (n_units < pre + P.l2_ahead ? n_units : pre + P.l2_ahead) : early;
     for (int it = 0; it < ahead; ++it) {
-      if (it < pre) {
+      if (it < early) {
         mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
         tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, kb * BK, row0);
       } else {
@@ -240,7 +241,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       tmW = tile_map(tile, row0);
       for (int it = 0; it < pre; ++it) {
         unsigned char *xd = tiles + (size_t)it * stage_bytes + W_STAGE_BYTES;
-        if (!P.early_w) {
+        if (it >= P.early_w) {
           mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
           tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, kb * BK, row0);
         }
@@ -387,6 +388,7 @@ int g_tune_max_split = 0;   // 0 = default rule
 int g_tune_no_streamk = 0;  // 1 = always the per-tile decomposition
 int g_tune_l2_ahead = -1;   // < 0 = default
 int g_tune_late_w = 0;      // 1 = weights wait for the dependency too
+int g_tune_early_stages = -1; // < 0 = all stages
 int g_tune_traffic_div = 8; // split <= K_in / (div * tokens)
 
 bool get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out) {
@@ -443,6 +445,7 @@ void tc_set_tuning(int key, int value) {
   if (key == 3) g_tune_no_streamk = value;
   if (key == 5) g_tune_l2_ahead = value;
   if (key == 6) g_tune_late_w = value;
+  if (key == 8) g_tune_early_stages = value;
   if (key == 7 && value > 0) g_tune_traffic_div = value;
 }
 
@@ -574,7 +577,7 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   if (stages < 2) return cudaErrorInvalidValue;
   P.stages = stages;
   P.l2_ahead = g_tune_l2_ahead >= 0 ? g_tune_l2_ahead : L2_AHEAD;
-  P.early_w = g_tune_late_w ? 0 : 1;
+  P.early_w = g_tune_late_w ? 0 : (g_tune_early_stages >= 0 && g_tune_early_stages < stages ? g_tune_early_stages : stages);
   CUtensorMap mw[3], mx, mxlo;
   for (int i = 0; i < 3; ++i) {
     const int j = i < m.n ? i : 0;
