@@ -139,8 +139,9 @@ cudaError_t eagle_concat(Launch L, int dtype, const float *feat_src, const int32
 // chunks of 1024 columns (chunks = ceil(H / 1024)).  H % 4 == 0.
 cudaError_t row_update(Launch L, int dtype, float *x, SplitIn P, const void *g, Operand xg, float *sumsq,
                        int R, int H);
+// q_out: rotated queries in fp32; q_pair (bf16 only, may be null): the same as a bf16 pair
 cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowScale sc, RowPlan plan, float *q_out,
-                          void *k_cache, void *v_cache, int R, int rows_per_seq, int n_heads,
+                          Operand q_pair, void *k_cache, void *v_cache, int R, int rows_per_seq, int n_heads,
                           int head_dim, int S_max);
 cudaError_t swiglu(Launch L, int dtype, SplitIn gu, RowScale sc, Operand act, int R, int F);
 cudaError_t tree_attention(Launch L, int dtype, const float *q, const void *k_cache,
@@ -159,6 +160,14 @@ size_t attn_mma_scratch_floats(int rows_total, int n_heads, int chunks);
 cudaError_t tree_attention_mma(Launch L, const float *q, const void *k_cache, const void *v_cache,
                                RowPlan plan, Operand out, float *scratch, int rows_per_seq, int B,
                                int n_heads, int S_max, int chunks);
+
+// attn_tc.cu : the same on tcgen05 tensor cores, all rows of a sequence in one CTA, key chunks as a cluster;
+// the queries come as the bf16 pair written by rope_kv_write ([q_rows_alloc][n_heads * 128] each)
+int attn_tc_chunks(int B, int n_heads, int S_max, int num_sms);
+bool attn_tc_supported(int rows_per_seq, int head_dim, int S_max);
+cudaError_t tree_attention_tc(Launch L, Operand q_pair, int q_rows_alloc, const void *k_cache, const void *v_cache,
+                              RowPlan plan, Operand out, int rows_per_seq, int B, int n_heads, int S_max, int chunks,
+                              int *status);
 
 // gemm_simt.cu : Y[R][sum n_out] (fp32, ld ldy) = X[R][K_in] * W^T, X and W of `dtype`
 cudaError_t gemm_simt(Launch L, int dtype, Operand X, GemmMats m, int K_in, int R, float *Y,

@@ -62,6 +62,7 @@ struct koala_ctx {
   int attn_chunks;
   float *x, *qbuf, *P, *verify_logits, *draft_logits, *verify_hid, *feat[2], *mx;
   Operand xn, attn_out, act, cat, lmin;
+  Operand qpair;           // rotated queries as a bf16 pair (bf16 configurations)
   bool pair;              // bf16 activations kept as hi + lo
   int32_t *verify_tgt, *s_parent, *s_level, *s_rank;
   int *status;
@@ -167,6 +168,11 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
   };
   c->xn = operand(H);
   c->attn_out = operand(H);
+  c->qpair = Operand{nullptr, nullptr};
+  if (cfg.dtype == KOALA_BF16) {
+    c->qpair.hi = w.take<unsigned char>((size_t)Mp * H * esz);
+    c->qpair.lo = w.take<unsigned char>((size_t)Mp * H * esz);
+  }
   c->act = operand(F);
   c->cat = operand(2 * H);
   c->lmin = operand(H);
@@ -295,11 +301,15 @@ int run_layer(koala_ctx *c, const LayerW &w, void *kc, void *vc, int R, int rows
   SplitIn s;
   GemmMats qkv{{w.wq, w.wk, w.wv}, {H, H, H}, 3};
   K_TRY(do_gemm(c, c->xn, H, qkv, R, nullptr, 0, &s));
-  CU_TRY(rope_kv_write(LN(c), g.dtype, s, c->pending, row_plan(c), c->qbuf, kc, vc, R, rows_per_seq, g.n_heads,
+  CU_TRY(rope_kv_write(LN(c), g.dtype, s, c->pending, row_plan(c), c->qbuf, c->qpair, kc, vc, R, rows_per_seq, g.n_heads,
                        g.head_dim, g.S_max));
   c->pending = none;
   const int ta = time_begin(c, KOALA_CLS_ATTENTION, 0);
-  if (c->use_tc && g.head_dim == 128 && c->attn_part != nullptr && rows_per_seq <= 128) {
+  if (c->use_tc && g.dtype == KOALA_BF16 && c->qpair.lo != nullptr &&
+      attn_tc_supported(rows_per_seq, g.head_dim, g.S_max)) {
+    CU_TRY(tree_attention_tc(LN(c), c->qpair, c->Mp, kc, vc, row_plan(c), c->attn_out, rows_per_seq, g.B, g.n_heads,
+                             g.S_max, attn_tc_chunks(g.B, g.n_heads, g.S_max, 148), c->status));
+  } else if (c->use_tc && g.head_dim == 128 && c->attn_part != nullptr && rows_per_seq <= 128) {
     CU_TRY(tree_attention_mma(LN(c), c->qbuf, kc, vc, row_plan(c), c->attn_out, c->attn_part, rows_per_seq,
                               g.B, g.n_heads, g.S_max,
                               attn_mma_chunks(g.B, g.n_heads, rows_per_seq, g.S_max, 148)));

@@ -265,6 +265,7 @@ __global__ void reduce_splits_kernel(SplitIn P, float *__restrict__ Y, int ldy, 
 // grid (R, n_heads), block head_dim/2: thread i rotates the pair (i, i + head_dim/2).
 template <typename T>
 __global__ void rope_kv_kernel(SplitIn qkv, RowScale sc, RowPlan plan, float *__restrict__ q_out,
+                               bf16 *__restrict__ qp_hi, bf16 *__restrict__ qp_lo,
                                T *__restrict__ k_cache, T *__restrict__ v_cache, int rows_per_seq,
                                int n_heads, int head_dim, int S_max) {
   pdl_launch_dependents();
@@ -277,8 +278,13 @@ __global__ void rope_kv_kernel(SplitIn qkv, RowScale sc, RowPlan plan, float *__
   const int c0 = h * head_dim + i, c1 = c0 + half;
   const float rs = sc.of(r);
   const float q0 = rs * qkv.at(r, c0), q1 = rs * qkv.at(r, c1);
-  q_out[(size_t)r * H + c0] = q0 * cs.x - q1 * cs.y;
-  q_out[(size_t)r * H + c1] = q1 * cs.x + q0 * cs.y;
+  const float qr0 = q0 * cs.x - q1 * cs.y, qr1 = q1 * cs.x + q0 * cs.y;
+  q_out[(size_t)r * H + c0] = qr0;
+  q_out[(size_t)r * H + c1] = qr1;
+  if (qp_hi != nullptr) {
+    store_operand(qp_hi, qp_lo, (size_t)r * H + c0, qr0);
+    store_operand(qp_hi, qp_lo, (size_t)r * H + c1, qr1);
+  }
   if (slot < 0 || slot >= S_max) return;
   const float k0 = rs * qkv.at(r, H + c0), k1 = rs * qkv.at(r, H + c1);
   const float v0 = rs * qkv.at(r, 2 * H + c0), v1 = rs * qkv.at(r, 2 * H + c1);
@@ -307,8 +313,9 @@ __device__ __forceinline__ void store2(bf16 *p, float a, float b) {
 }
 template <typename T>
 __global__ void __launch_bounds__(1024)
-rope_kv_vec_kernel(SplitIn qkv, RowScale sc, RowPlan plan, float *__restrict__ q_out, T *__restrict__ k_cache,
-                   T *__restrict__ v_cache, int rows_per_seq, int n_heads, int head_dim, int S_max) {
+rope_kv_vec_kernel(SplitIn qkv, RowScale sc, RowPlan plan, float *__restrict__ q_out, bf16 *__restrict__ qp_hi,
+                   bf16 *__restrict__ qp_lo, T *__restrict__ k_cache, T *__restrict__ v_cache, int rows_per_seq,
+                   int n_heads, int head_dim, int S_max) {
   pdl_launch_dependents();
   pdl_wait();
   const int r = blockIdx.x;
@@ -324,8 +331,18 @@ rope_kv_vec_kernel(SplitIn qkv, RowScale sc, RowPlan plan, float *__restrict__ q
     const int c0 = h * head_dim + i, c1 = c0 + half;
     float2 qa = split_sum2(qkv, r, c0), qb = split_sum2(qkv, r, c1);
     qa.x *= rs; qa.y *= rs; qb.x *= rs; qb.y *= rs;
-    store2(q_out + (size_t)r * H + c0, qa.x * cs.x - qb.x * cs.y, qa.y * cs.z - qb.y * cs.w);
-    store2(q_out + (size_t)r * H + c1, qb.x * cs.x + qa.x * cs.y, qb.y * cs.z + qa.y * cs.w);
+    const float2 ra = make_float2(qa.x * cs.x - qb.x * cs.y, qa.y * cs.z - qb.y * cs.w);
+    const float2 rb = make_float2(qb.x * cs.x + qa.x * cs.y, qb.y * cs.z + qa.y * cs.w);
+    store2(q_out + (size_t)r * H + c0, ra.x, ra.y);
+    store2(q_out + (size_t)r * H + c1, rb.x, rb.y);
+    if (qp_hi != nullptr) {      // the same values as a bf16 pair (value + rounding residual)
+      const __nv_bfloat162 ha = __floats2bfloat162_rn(ra.x, ra.y), hb = __floats2bfloat162_rn(rb.x, rb.y);
+      const float2 fa = __bfloat1622float2(ha), fb = __bfloat1622float2(hb);
+      *reinterpret_cast<__nv_bfloat162 *>(qp_hi + (size_t)r * H + c0) = ha;
+      *reinterpret_cast<__nv_bfloat162 *>(qp_hi + (size_t)r * H + c1) = hb;
+      *reinterpret_cast<__nv_bfloat162 *>(qp_lo + (size_t)r * H + c0) = __floats2bfloat162_rn(ra.x - fa.x, ra.y - fa.y);
+      *reinterpret_cast<__nv_bfloat162 *>(qp_lo + (size_t)r * H + c1) = __floats2bfloat162_rn(rb.x - fb.x, rb.y - fb.y);
+    }
     if (!wr) continue;
     float2 ka = split_sum2(qkv, r, H + c0), kb = split_sum2(qkv, r, H + c1);
     float2 va = split_sum2(qkv, r, 2 * H + c0), vb = split_sum2(qkv, r, 2 * H + c1);
@@ -582,18 +599,20 @@ cudaError_t row_update(Launch L, int dtype, float *x, SplitIn P, const void *g, 
 }
 
 cudaError_t rope_kv_write(Launch L, int dtype, SplitIn qkv, RowScale sc, RowPlan plan, float *q_out,
-                          void *k_cache, void *v_cache, int R, int rows_per_seq, int n_heads,
+                          Operand q_pair, void *k_cache, void *v_cache, int R, int rows_per_seq, int n_heads,
                           int head_dim, int S_max) {
+  bf16 *qh = (bf16 *)q_pair.hi, *ql = (bf16 *)q_pair.lo;
+  if (dtype == 0 || ql == nullptr) qh = ql = nullptr;      // the pair exists for bf16 storage only
   if (head_dim % 4 == 0 && qkv.ld % 2 == 0 && qkv.stride % 2 == 0) {
     const int work = n_heads * head_dim / 4;
     const int threads = work < 128 ? ((work + 31) / 32) * 32 : 128;
     const int slices = (work + threads - 1) / threads;
     DISPATCH_T(dtype, return launch_k(rope_kv_vec_kernel<T>, dim3(R, slices), dim3(threads), 0, L.st, L.pdl, qkv, sc, plan,
-                                      q_out, (T *)k_cache, (T *)v_cache, rows_per_seq, n_heads, head_dim,
+                                      q_out, qh, ql, (T *)k_cache, (T *)v_cache, rows_per_seq, n_heads, head_dim,
                                       S_max);)
   }
   DISPATCH_T(dtype, return launch_k(rope_kv_kernel<T>, dim3(R, n_heads), dim3(head_dim / 2), 0, L.st,
-                                    L.pdl, qkv, sc, plan, q_out, (T *)k_cache, (T *)v_cache,
+                                    L.pdl, qkv, sc, plan, q_out, qh, ql, (T *)k_cache, (T *)v_cache,
                                     rows_per_seq, n_heads, head_dim, S_max);)
 }
 
