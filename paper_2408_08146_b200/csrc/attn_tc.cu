@@ -10,14 +10,15 @@
 // and the rows fold O_t into their running (max, sum, O) in registers.  Q and P enter the MMAs as
 // bf16 pairs (value + rounding residual: two accumulating MMAs), so only the cached K and V carry
 // bf16 rounding.  Q (written as a pair by the rotary-embedding kernel) and the K/V tiles arrive by
-// TMA with the 128-byte swizzle, K/V in a three-stage ring; S and O_t are double-buffered in tensor
-// memory, P in shared memory, so the tensor pipe works on tile t+1 while the rows process tile t.
+// TMA with the 128-byte swizzle, K/V in a two-stage ring; S is double-buffered in tensor memory, so
+// the tensor pipe computes the scores of tile t+1 while the rows process tile t.
 // Warps 0..3 own the rows, warp 4 lane 0 issues the copies, warp 5 lane 0 the MMAs.
-// With several chunks the CTAs of one (head, sequence) form a thread-block cluster: after a
-// cluster barrier every CTA pushes, into each peer's shared memory, that peer's slice of the head
-// dimension of its unnormalised (O, m, l); after a second barrier every CTA merges its slice over
-// the chunks in chunk order from its own shared memory and writes it as a matrix-multiply operand
-// pair.
+// With several chunks the CTAs of one (head, sequence) form a thread-block cluster: every CTA
+// pushes, into each peer's shared memory, that peer's slice of the head dimension of its
+// unnormalised (O, m, l); after a cluster barrier every CTA merges its slice over the chunks in
+// chunk order from its own shared memory and writes it as a matrix-multiply operand pair.  (With
+// more than 64 rows the receive buffer reuses the K/V ring, so a first cluster barrier makes sure
+// that every peer is done with its tiles.)
 // The mask is: slots below ctx_len visible to every row; slot ctx_len + j visible to a row iff
 // bit j of its 128-bit mask; slots from kv_len on invisible.
 // Every wait is bounded: on expiry the kernel records a timeout in *status and returns.
@@ -33,21 +34,25 @@ namespace {
 
 constexpr int DH = 128;
 constexpr int TK = 64;                       // keys per tile
-constexpr int NKV = 3;                       // K/V stages
+constexpr int NKV = 2;                       // K/V stages
 constexpr int SUB = 64 * 64 * 2;             // one [64 keys][64 dims] block: 8 KB
 constexpr int QSUB = 128 * 64 * 2;           // one [128 rows][64 columns] block: 16 KB
 constexpr int OFF_Q = 0;                     // Q hi (2 blocks), Q lo (2 blocks)
 constexpr int OFF_KV = 4 * QSUB;             // stages of K (2 blocks) + V (2 blocks)
 constexpr int KV_STAGE = 4 * SUB;
-constexpr int OFF_P = OFF_KV + NKV * KV_STAGE;   // 2 buffers of P hi, P lo
+constexpr int OFF_P = OFF_KV + NKV * KV_STAGE;   // P hi, P lo
 constexpr int P_BUF = 2 * QSUB;
-constexpr int SMEM_BYTES = OFF_P + 2 * P_BUF;    // 224 KB
+constexpr int OFF_RECV = OFF_P + P_BUF;          // chunk-merge buffer when at most 64 rows are in use
+constexpr int RECV_BYTES = 8 * 64 * (DH / 8 + 4) * 4;
+constexpr int SMEM_BYTES = OFF_RECV + RECV_BYTES;    // 200 KB
 constexpr int THREADS = 192;
 constexpr int E_TIMEOUT = 6;
-constexpr int TMEM_COLS = 512;               // S: 2 x 64 columns, O_t: 2 x 128 columns
+constexpr int TMEM_COLS = 256;               // S: 2 x 64 columns, O_t: 128 columns
 constexpr int COL_S = 0, COL_O = 128;
-static_assert(8 * 128 * (DH / 8 + 4) * 4 <= NKV * KV_STAGE && 128 * (DH + 4) * 4 <= NKV * KV_STAGE,
-              "the chunk-merge buffer fits in the K/V ring");
+static_assert(8 * 128 * (DH / 8 + 4) * 4 <= NKV * KV_STAGE + P_BUF && 128 * (DH + 4) * 4 <= NKV * KV_STAGE + P_BUF,
+              "with more than 64 rows the chunk-merge buffer fits in the K/V ring plus P");
+static_assert(64 * (DH + 4) * 4 <= RECV_BYTES && 2 * 64 * (DH / 2 + 4) * 4 <= RECV_BYTES && 4 * 64 * (DH / 4 + 4) * 4 <= RECV_BYTES,
+              "with at most 64 rows the chunk-merge buffer has room of its own");
 
 __device__ __forceinline__ void split_pack(float x, float y, uint32_t &hi, uint32_t &lo) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
@@ -112,7 +117,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   constexpr int NC = DUP ? 32 : 64;      // score columns (keys of a tile) per thread
   constexpr int ND = DUP ? 64 : 128;     // output dims per thread
   extern __shared__ unsigned char smem_raw[];
-  __shared__ uint64_t q_full, kv_full[NKV], kv_empty[NKV], s_full[2], p_full[2], o_full[2], x_bar[2];
+  __shared__ uint64_t q_full, kv_full[NKV], kv_empty[NKV], s_full[2], p_full, o_full, x_bar[2];
   __shared__ float xch[2][128];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int s_error;
@@ -131,10 +136,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   if (threadIdx.x == 0) {
     mbar_init(&q_full, 1);
     for (int s = 0; s < NKV; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+    mbar_init(&p_full, (uint32_t)n_arrive);
+    mbar_init(&o_full, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s_full[i], 1);
-      mbar_init(&p_full[i], (uint32_t)n_arrive);
-      mbar_init(&o_full[i], 1);
       mbar_init(&x_bar[i], 2);
     }
     s_error = 0;
@@ -156,6 +161,17 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   const uint32_t tmem = tmem_base_slot;
 
   pdl_wait();                      // Q, the tree rows of K/V and the row plan come from earlier kernels
+  if (threadIdx.x == 128) {        // warp 4 lane 0: the queries do not depend on the plan
+    mbar_expect_tx(&q_full, (uint32_t)(4 * QSUB));
+#pragma unroll
+    for (int part = 0; part < 2; ++part)
+#pragma unroll
+      for (int hb = 0; hb < 2; ++hb)
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh)
+          tma_load_2d(part ? &tmQl : &tmQh, &q_full, sm + OFF_Q + (part * 2 + hb) * QSUB + rh * (QSUB / 2),
+                      h * DH + 64 * hb, b * P.rows_per_seq + (DUP ? 0 : 64 * rh));
+  }
   const int ctx = P.plan.ctx_len[b];
   int kv_len = P.plan.kv_len[b];
   kv_len = kv_len > P.S_max ? P.S_max : kv_len;
@@ -177,15 +193,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   if (warp == 4) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      mbar_expect_tx(&q_full, (uint32_t)(4 * QSUB));
-#pragma unroll
-      for (int part = 0; part < 2; ++part)
-#pragma unroll
-        for (int hb = 0; hb < 2; ++hb)
-#pragma unroll
-          for (int rh = 0; rh < 2; ++rh)
-            tma_load_2d(part ? &tmQl : &tmQh, &q_full, sm + OFF_Q + (part * 2 + hb) * QSUB + rh * (QSUB / 2),
-                        h * DH + 64 * hb, b * P.rows_per_seq + (DUP ? 0 : 64 * rh));
       const int y0 = (b * P.n_heads + h) * P.S_max;
       bool ok = true;
       int issued = 0;
@@ -243,12 +250,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       if (ok && T > 0) ok = issue_s(0);
       for (int t = 0; t < T && ok; ++t) {
         if (t + 1 < T) { ok = issue_s(t + 1); if (!ok) break; }
-        ok = mbar_wait(&p_full[t & 1], (uint32_t)(t >> 1) & 1u);
+        ok = mbar_wait(&p_full, (uint32_t)t & 1u);
         if (!ok) break;
         tc_fence_after();
         const uint32_t vb = sb + OFF_KV + (t % NKV) * KV_STAGE + 2 * SUB;
-        const uint32_t pb = sb + OFF_P + (t & 1) * P_BUF;
-        const uint32_t d = tmem + (uint32_t)(COL_O + (t & 1) * DH);
+        const uint32_t pb = sb + OFF_P;
+        const uint32_t d = tmem + (uint32_t)COL_O;
 #pragma unroll
         for (int part = 0; part < 2; ++part) {            // P value, then P residual
           const uint64_t da = smem_desc_sw128(pb + part * QSUB);
@@ -259,7 +266,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
           }
         }
         umma_commit(&kv_empty[t % NKV]);
-        umma_commit(&o_full[t & 1]);
+        umma_commit(&o_full);
       }
       if (!ok) atomicExch(&s_error, 1);
     }
@@ -279,14 +286,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     float m_prev = -INFINITY, l_prev = 0.f;
 
     auto merge_o = [&](int u, float m_u, float l_u) -> bool {
-      if (!__all_sync(0xffffffffu, mbar_wait(&o_full[u & 1], (uint32_t)(u >> 1) & 1u))) return false;
+      if (!__all_sync(0xffffffffu, mbar_wait(&o_full, (uint32_t)u & 1u))) return false;
       tc_fence_after();
       const float m_new = fmaxf(m_run, m_u);
       const float mu = m_new == -INFINITY ? 0.f : m_new;
       const float a = exp2f(m_run - mu), bw = exp2f(m_u - mu);      // exp2(-inf) = 0
       l_run = l_run * a + l_u * bw;
       m_run = m_new;
-      const uint32_t base = tmem + lane_sel + (uint32_t)(COL_O + (u & 1) * DH + ND * half);
+      const uint32_t base = tmem + lane_sel + (uint32_t)(COL_O + ND * half);
 #pragma unroll
       for (int c0 = 0; c0 < ND; c0 += 32) {
         uint32_t v[32];
@@ -327,9 +334,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         if (!ok) break;
         m_t = fmaxf(m_t, xch[t & 1][threadIdx.x ^ 64]);
       }
+      // fold the previous tile's P V in first: that also tells that P and O_t may be overwritten
+      if (t >= 1) {
+        ok = merge_o(t - 1, m_prev, l_prev);
+        if (!ok) break;
+      }
       const float mu = m_t == -INFINITY ? 0.f : m_t;
       float l_t = 0.f;
-      const uint32_t pb = sb + OFF_P + (t & 1) * P_BUF + prow;
+      const uint32_t pb = sb + OFF_P + prow;
 #pragma unroll
       for (int ch = 0; ch < NC / 8; ++ch) {
         uint32_t hi[4], lo[4];
@@ -351,11 +363,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full[t & 1]);
-      if (t >= 1) {
-        ok = merge_o(t - 1, m_prev, l_prev);
-        if (!ok) break;
-      }
+      if (lane == 0) mbar_arrive(&p_full);
       m_prev = m_t;
       l_prev = l_t;
     }
@@ -364,16 +372,17 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   }
 
   tc_fence_before();
-  __syncthreads();                       // all tiles consumed: the K/V ring is free for the merge buffer
+  __syncthreads();                       // all tiles consumed
   const bool failed = s_error != 0;
   // ---- merge over the chunks.  Every CTA receives, from every chunk j (itself included), the
-  // dims [c * wc, (c + 1) * wc) of all rows plus (m, l): recv[j][row][wc + 4] in its K/V ring.
+  // dims [c * wc, (c + 1) * wc) of all rows plus (m, l): recv[j][row][wc + 4].
   const int wc = DH / P.chunks;
   const int rs = wc + 4;                 // floats per received row: wc dims, m, l (first keys), l (other keys), pad
-  float *recv = reinterpret_cast<float *>(sm + OFF_KV);
-  if (P.chunks > 1) cluster_sync_all();  // every CTA of the cluster is done with its K/V ring
+  constexpr int RR = DUP ? 64 : 128;     // rows per source chunk in the receive buffer
+  float *recv = reinterpret_cast<float *>(sm + (DUP ? OFF_RECV : OFF_KV));
+  if (!DUP && P.chunks > 1) cluster_sync_all();  // every CTA of the cluster is done with its K/V ring
   if (row_in) {
-    const uint32_t mine = smem_u32(recv + ((size_t)c * 128 + row) * rs);
+    const uint32_t mine = smem_u32(recv + ((size_t)c * RR + row) * rs);
 #pragma unroll
     for (int d = 0; d < ND; d += 4) {
       const int gd = ND * half + d;
@@ -394,14 +403,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     const int ncol = DUP ? wc / 2 : wc;                    // this thread's share of the CTA's dims
     const int col0 = DUP ? half * ncol : 0;
     float mm = -INFINITY;
-    for (int j = 0; j < P.chunks; ++j) mm = fmaxf(mm, recv[((size_t)j * 128 + row) * rs + wc]);
+    for (int j = 0; j < P.chunks; ++j) mm = fmaxf(mm, recv[((size_t)j * RR + row) * rs + wc]);
     float o[ND];
 #pragma unroll
     for (int d = 0; d < ND; ++d) o[d] = 0.f;
     float l = 0.f;
     if (mm != -INFINITY) {
       for (int j = 0; j < P.chunks; ++j) {
-        const float *src = recv + ((size_t)j * 128 + row) * rs;
+        const float *src = recv + ((size_t)j * RR + row) * rs;
         const float4 ml = *reinterpret_cast<const float4 *>(src + wc);
         if (ml.x == -INFINITY) continue;
         const float w = exp2f(ml.x - mm);
