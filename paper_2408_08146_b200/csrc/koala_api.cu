@@ -143,7 +143,8 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
   int draft_rows = B * k;
   if (cfg.head_kind == KOALA_MEDUSA && cfg.n_medusa_heads * B > draft_rows) draft_rows = cfg.n_medusa_heads * B;
   int rows = M > draft_rows ? M : draft_rows;
-  const int Mp = (int)align_up((size_t)rows + 16, 16);
+  // padded row count: the tensor-core GEMM reads whole token tiles (up to 256 rows) of its input
+  const int Mp = (int)align_up((size_t)rows + 16, rows > 128 ? 256 : 16);
   const int pool = cfg.head_kind == KOALA_EAGLE ? k + (cfg.D - 1) * k * k : k;
   const size_t pcols = (size_t)(3 * H > 2 * F ? 3 * H : 2 * F);
   const size_t esz = cfg.dtype == KOALA_FP32 ? 4 : 2;

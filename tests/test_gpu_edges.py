@@ -114,6 +114,41 @@ def test_long_context_many_key_tiles_and_chunks(context):
     eng.close()
 
 
+@pytest.mark.parametrize("N,B,n_heads,context,S_max", [
+    (128, 1, 32, 1000, 4096),    # more than 64 rows: every row warp owns its rows; 4 key chunks
+    (100, 2, 32, 700, 1024),     # ragged row count above 64, 2 chunks, two sequences
+    (20, 1, 32, 300, 512),       # fewer than 32 rows: one row group, duplicated
+    (40, 8, 32, 200, 512),       # more CTAs than SMs: a single chunk, no cluster
+    (60, 1, 8, 3000, 4096),      # few heads: 8 key chunks per head
+    (33, 1, 32, 64, 256),        # context shorter than a chunk's share: empty chunks
+])
+def test_tensor_core_attention_shapes(N, B, n_heads, context, S_max):
+    """One bf16 layer with head_dim 128 at row counts, batch sizes and chunk counts that select
+    every variant of the tcgen05 attention kernel; the tree sits on top of a random cache."""
+    H = n_heads * 128
+    cfg = reduced(T7_EAGLE, 1, K=1, N=N, B=B, H=H, n_heads=n_heads, F=2 * H, V=2048, D=min(5, N - 1),
+                  S_max=S_max, prompt_len=context)
+    eng, orc, _ = make_pair(cfg, oracle_dtype=np.float32, cache_host=False)
+    eng.target_k.copy_(random_kv(cfg, "target_k", cfg.L, DEV))
+    eng.target_v.copy_(random_kv(cfg, "target_v", cfg.L, DEV))
+    lens = [context - 13 * b for b in range(B)]
+    for b in range(B):
+        orc.target_k[0][b][...] = kv_to_oracle(eng.target_k, 0, b, np.float32)
+        orc.target_v[0][b][...] = kv_to_oracle(eng.target_v, 0, b, np.float32)
+        orc.seq_len[b] = lens[b]
+    eng.seq_len.copy_(torch.tensor(lens, dtype=torch.int32))
+    par = [-1] + [max(0, u - 1 - (u * 7) % min(u, 5)) for u in range(1, N)]
+    toks = [uniform_ints(11 + b, "edge.shapes", N, 0, cfg.V) for b in range(B)]
+    eng.koala_verify(_tree_arrays(eng, toks, [par] * B))
+    orc.verify([(toks[b], np.asarray(par)) for b in range(B)])
+    bufs = eng.buffers()
+    for b in range(B):
+        assert_close(bufs["verify_hid"][b * N:(b + 1) * N].cpu().numpy(), orc.verify_hid[b], cfg.dtype,
+                     f"hidden, sequence {b}")
+    assert eng.device_status() == 0
+    eng.close()
+
+
 def test_capacity_and_malformed_trees_are_reported_not_executed():
     cfg = TINY_EAGLE.with_(S_max=80)                    # the 64-token prompt fits, prompt + tree does not
     eng, orc, _ = make_pair(cfg)
