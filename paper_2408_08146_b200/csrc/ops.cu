@@ -92,13 +92,24 @@ __global__ void row_epilogue_kernel(int mode, float *__restrict__ x, SplitIn P,
 // Vectorised variant for H % 4 == 0: one CTA per row, every thread owns up to VPT groups of four
 // consecutive columns, keeps them in registers between the two passes and issues all split-K
 // partial loads of a group back to back.
+// (The first eight partial loads are issued before any is used - one trip to L2 instead of one
+// per partial; the additions keep the slot order.)
+template <int AHEAD = 8>
 __device__ __forceinline__ float4 split_sum4(const SplitIn &P, int r, int c) {
   const float *q = P.p + (size_t)r * P.ld + c;
-  float4 v = *reinterpret_cast<const float4 *>(q);
   const int k = P.count(c);
-  for (int s = 1; s < k; ++s) {
-    const float4 u = *reinterpret_cast<const float4 *>(q + (size_t)s * P.stride);
-    v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
+  float4 u[AHEAD];
+#pragma unroll
+  for (int s = 0; s < AHEAD; ++s)
+    u[s] = s < k ? *reinterpret_cast<const float4 *>(q + (size_t)s * P.stride) : make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 v = u[0];
+#pragma unroll
+  for (int s = 1; s < AHEAD; ++s) {
+    if (s < k) { v.x += u[s].x; v.y += u[s].y; v.z += u[s].z; v.w += u[s].w; }
+  }
+  for (int s = AHEAD; s < k; ++s) {
+    const float4 w = *reinterpret_cast<const float4 *>(q + (size_t)s * P.stride);
+    v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
   }
   return v;
 }
@@ -299,11 +310,19 @@ __global__ void rope_kv_kernel(SplitIn qkv, RowScale sc, RowPlan plan, float *__
 // one head with 8-byte loads.
 __device__ __forceinline__ float2 split_sum2(const SplitIn &P, int r, int c) {
   const float *q = P.p + (size_t)r * P.ld + c;
-  float2 v = *reinterpret_cast<const float2 *>(q);
   const int k = P.count(c);
-  for (int s = 1; s < k; ++s) {
-    const float2 u = *reinterpret_cast<const float2 *>(q + (size_t)s * P.stride);
-    v.x += u.x; v.y += u.y;
+  float2 u[4];
+#pragma unroll
+  for (int s = 0; s < 4; ++s)
+    u[s] = s < k ? *reinterpret_cast<const float2 *>(q + (size_t)s * P.stride) : make_float2(0.f, 0.f);
+  float2 v = u[0];
+#pragma unroll
+  for (int s = 1; s < 4; ++s) {
+    if (s < k) { v.x += u[s].x; v.y += u[s].y; }
+  }
+  for (int s = 4; s < k; ++s) {
+    const float2 w = *reinterpret_cast<const float2 *>(q + (size_t)s * P.stride);
+    v.x += w.x; v.y += w.y;
   }
   return v;
 }
@@ -329,7 +348,10 @@ rope_kv_vec_kernel(SplitIn qkv, RowScale sc, RowPlan plan, float *__restrict__ q
     const int h = p / hq, i = (p - h * hq) * 2;
     const float4 cs = *reinterpret_cast<const float4 *>(&plan.rope[(size_t)r * half + i]);   // c0 s0 c1 s1
     const int c0 = h * head_dim + i, c1 = c0 + half;
+    // all partial sums of this thread are requested before the first store
     float2 qa = split_sum2(qkv, r, c0), qb = split_sum2(qkv, r, c1);
+    float2 ka = split_sum2(qkv, r, H + c0), kb = split_sum2(qkv, r, H + c1);
+    float2 va = split_sum2(qkv, r, 2 * H + c0), vb = split_sum2(qkv, r, 2 * H + c1);
     qa.x *= rs; qa.y *= rs; qb.x *= rs; qb.y *= rs;
     const float2 ra = make_float2(qa.x * cs.x - qb.x * cs.y, qa.y * cs.z - qb.y * cs.w);
     const float2 rb = make_float2(qb.x * cs.x + qa.x * cs.y, qb.y * cs.z + qa.y * cs.w);
@@ -344,8 +366,6 @@ rope_kv_vec_kernel(SplitIn qkv, RowScale sc, RowPlan plan, float *__restrict__ q
       *reinterpret_cast<__nv_bfloat162 *>(qp_lo + (size_t)r * H + c1) = __floats2bfloat162_rn(rb.x - fb.x, rb.y - fb.y);
     }
     if (!wr) continue;
-    float2 ka = split_sum2(qkv, r, H + c0), kb = split_sum2(qkv, r, H + c1);
-    float2 va = split_sum2(qkv, r, 2 * H + c0), vb = split_sum2(qkv, r, 2 * H + c1);
     ka.x *= rs; ka.y *= rs; kb.x *= rs; kb.y *= rs;
     va.x *= rs; va.y *= rs; vb.x *= rs; vb.y *= rs;
     const size_t base = (((size_t)b * n_heads + h) * S_max + slot) * head_dim + i;
@@ -376,7 +396,7 @@ __global__ void swiglu_vec_kernel(SplitIn gu, RowScale sc, T *__restrict__ act, 
   const int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (f >= F) return;
   const float rs = sc.of(r);
-  const float4 a = split_sum4(gu, r, f), b = split_sum4(gu, r, F + f);
+  const float4 a = split_sum4<3>(gu, r, f), b = split_sum4<3>(gu, r, F + f);
   store_operand4(act, act_lo, (size_t)r * F + f,
                  make_float4(silu_f(rs * a.x) * (rs * b.x), silu_f(rs * a.y) * (rs * b.y),
                              silu_f(rs * a.z) * (rs * b.z), silu_f(rs * a.w) * (rs * b.w)));
