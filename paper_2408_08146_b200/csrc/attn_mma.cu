@@ -76,7 +76,7 @@ constexpr int NST = 3;                   // cp.async stages
 constexpr int MSTRIDE = DH + 4;          // floats per merged row in shared memory (keeps 16-byte alignment)
 
 __global__ void __launch_bounds__(128)
-tree_attn_mma_kernel(const float *__restrict__ q, const bf16 *__restrict__ kc, const bf16 *__restrict__ vc,
+tree_attn_mma_kernel(const float *q, const bf16 *kc, const bf16 *vc,
                      RowPlan plan, float *__restrict__ part, bf16 *__restrict__ out, bf16 *__restrict__ out_lo,
                      int rows_per_seq, int n_heads, int S_max, int chunks) {
   extern __shared__ __align__(1024) unsigned char smem[];     // [NST][K tile | V tile]
@@ -324,7 +324,7 @@ tree_attn_mma_kernel(const float *__restrict__ q, const bf16 *__restrict__ kc, c
 
 // One warp per (row, head): merges the chunk partials in chunk order and writes the operand pair.
 __global__ void __launch_bounds__(256)
-tree_attn_combine_kernel(const float *__restrict__ part, bf16 *__restrict__ out, bf16 *__restrict__ out_lo,
+tree_attn_combine_kernel(const float *part, bf16 *__restrict__ out, bf16 *__restrict__ out_lo,
                          int R, int n_heads, int chunks) {
   pdl_launch_dependents();
   pdl_wait();

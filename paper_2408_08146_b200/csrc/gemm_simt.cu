@@ -13,7 +13,7 @@ constexpr int WARPS = 8;
 
 template <typename T>
 __global__ void __launch_bounds__(WARPS * 32)
-gemm_simt_kernel(const T *__restrict__ X, const T *__restrict__ Xlo, int R, int K_in, const T *__restrict__ W0,
+gemm_simt_kernel(const T *X, const T *Xlo, int R, int K_in, const T *__restrict__ W0,
                  const T *__restrict__ W1, const T *__restrict__ W2, int n0, int n1, int n2,
                  float *__restrict__ Y, int ldy) {
   __shared__ float xs[ROWS][KC + 1];

@@ -37,7 +37,7 @@ __device__ __forceinline__ void store_operand(T *hi, T *lo, size_t i, float v) {
 
 // ------------------------------------------------------------------------------- embedding + norm
 template <typename T>
-__global__ void embed_norm_kernel(const int32_t *__restrict__ tok, const T *__restrict__ E,
+__global__ void embed_norm_kernel(const int32_t *tok, const T *__restrict__ E,
                                   const T *__restrict__ g, float *__restrict__ x,
                                   T *__restrict__ xn, T *__restrict__ xn_lo, int H, int V, float eps) {
   __shared__ float red[32];
@@ -229,9 +229,9 @@ row_update_kernel(float *__restrict__ x, SplitIn P, const T *__restrict__ g, T *
 
 // ------------------------------------------------------------------------------- EAGLE fc input
 template <typename T>
-__global__ void eagle_concat_kernel(const float *__restrict__ feat_src,
-                                    const int32_t *__restrict__ row_src,
-                                    const int32_t *__restrict__ row_tok, const T *__restrict__ E,
+__global__ void eagle_concat_kernel(const float *feat_src,
+                                    const int32_t *row_src,
+                                    const int32_t *row_tok, const T *__restrict__ E,
                                     T *__restrict__ cat, T *__restrict__ cat_lo, int H, int V) {
   pdl_launch_dependents();
   pdl_wait();
@@ -250,7 +250,7 @@ __global__ void eagle_concat_kernel(const float *__restrict__ feat_src,
 }
 
 template <typename T>
-__global__ void cast_rows_kernel(const float *__restrict__ src, const int32_t *__restrict__ row_src,
+__global__ void cast_rows_kernel(const float *src, const int32_t *row_src,
                                  T *__restrict__ dst, T *__restrict__ dst_lo,
                                  float *__restrict__ dst32, int dst32_stride, int H) {
   pdl_launch_dependents();
@@ -408,7 +408,7 @@ __global__ void swiglu_vec_kernel(SplitIn gu, RowScale sc, T *__restrict__ act, 
 // each lane owning DH/32 output dimensions.  Online softmax in fp32.
 template <typename T, int DH>
 __global__ void __launch_bounds__(256)
-tree_attn_kernel(const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc,
+tree_attn_kernel(const float *q, const T *kc, const T *vc,
                  RowPlan plan, T *__restrict__ out, T *__restrict__ out_lo, int rows_per_seq,
                  int n_heads, int S_max) {
   __shared__ float Ks[32][DH + 1];
@@ -509,7 +509,7 @@ __device__ __forceinline__ ValIdx block_argmax(ValIdx x, ValIdx *red) {
   return x;
 }
 
-__global__ void argmax_rows_kernel(const float *__restrict__ logits, int32_t *__restrict__ out, int V) {
+__global__ void argmax_rows_kernel(const float *logits, int32_t *__restrict__ out, int V) {
   __shared__ ValIdx red[32];
   pdl_launch_dependents();
   pdl_wait();
@@ -522,7 +522,7 @@ __global__ void argmax_rows_kernel(const float *__restrict__ logits, int32_t *__
 
 // Per row: the k largest logits (ties: smaller id) and their natural-log softmax probabilities.
 // The row is staged in shared memory; each round removes the current maximum.
-__global__ void topk_logp_kernel(const float *__restrict__ logits, int32_t *__restrict__ tok,
+__global__ void topk_logp_kernel(const float *logits, int32_t *__restrict__ tok,
                                  float *__restrict__ logp, int V, int k) {
   extern __shared__ float srow[];
   __shared__ ValIdx red[32];
@@ -553,6 +553,85 @@ __global__ void topk_logp_kernel(const float *__restrict__ logits, int32_t *__re
       srow[best.i] = -INFINITY;
     }
     __syncthreads();
+  }
+}
+
+__device__ __forceinline__ ValIdx warp_argmax(ValIdx x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    ValIdx y;
+    y.v = __shfl_xor_sync(0xffffffffu, x.v, o);
+    y.i = __shfl_xor_sync(0xffffffffu, x.i, o);
+    x = better(x, y);
+  }
+  return x;
+}
+
+// Same result for V <= 32768 and k <= 32 with two levels instead of k passes over the row: every
+// thread keeps its 32 strided elements in registers, every warp extracts the k best of its 1024
+// elements with shuffles only, and warp 0 extracts the k best of the 32 * k survivors.  (The k
+// best of the row are among the k best of each part; ties still go to the smaller id.)
+__global__ void __launch_bounds__(1024)
+topk_logp_fast_kernel(const float *logits, int32_t *__restrict__ tok, float *__restrict__ logp,
+                      int V, int k) {
+  __shared__ ValIdx cand[32 * 32];
+  __shared__ float redf[32];
+  __shared__ float s_mx;
+  pdl_launch_dependents();
+  pdl_wait();
+  const float *row = logits + (size_t)blockIdx.x * V;
+  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+  float vals[32];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    const int i = tid + 1024 * j;
+    vals[j] = i < V ? row[i] : -INFINITY;
+    mx = fmaxf(mx, vals[j]);
+  }
+  mx = warp_max(mx);
+  if (lane == 0) redf[w] = mx;
+  __syncthreads();
+  if (w == 0) {
+    const float m2 = warp_max(redf[lane]);
+    if (lane == 0) s_mx = m2;
+  }
+  __syncthreads();
+  mx = s_mx;
+  float se = 0.f;
+#pragma unroll
+  for (int j = 0; j < 32; ++j) se += expf(vals[j] - mx);       // exp(-inf) = 0 for the padding
+  const float lse = mx + logf(block_sum(se, redf));
+  for (int r = 0; r < k; ++r) {
+    ValIdx best{-INFINITY, 0x7fffffff};
+#pragma unroll
+    for (int j = 0; j < 32; ++j) best = better(best, ValIdx{vals[j], tid + 1024 * j});
+    best = warp_argmax(best);
+    if ((best.i & 1023) == tid) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j == (best.i >> 10)) vals[j] = -INFINITY;
+    }
+    if (lane == 0) cand[w * k + r] = best;
+  }
+  __syncthreads();
+  if (w == 0) {
+    const int n = 32 * k;
+    for (int r = 0; r < k; ++r) {
+      ValIdx best{-INFINITY, 0x7fffffff};
+      int at = -1;
+      for (int c = lane; c < n; c += 32) {
+        const ValIdx x = cand[c];
+        if (x.v > best.v || (x.v == best.v && x.i < best.i)) { best = x; at = c; }
+      }
+      const ValIdx win = warp_argmax(best);
+      if (at >= 0 && best.i == win.i) cand[at] = ValIdx{-INFINITY, 0x7fffffff};
+      __syncwarp();
+      if (lane == 0) {
+        tok[(size_t)blockIdx.x * k + r] = win.i;
+        logp[(size_t)blockIdx.x * k + r] = win.v - lse;
+      }
+    }
   }
 }
 
@@ -667,6 +746,8 @@ cudaError_t argmax_rows(Launch L, const float *logits, int32_t *out, int R, int 
 }
 
 cudaError_t topk_logp(Launch L, const float *logits, int32_t *tok, float *logp, int R, int V, int k) {
+  if (V <= 32768 && k <= 32)
+    return launch_k(topk_logp_fast_kernel, dim3(R), dim3(1024), 0, L.st, L.pdl, logits, tok, logp, V, k);
   const size_t smem = (size_t)V * sizeof(float);
   static size_t configured = 0;
   if (smem > 48 * 1024 && smem > configured) {

@@ -25,9 +25,9 @@ __device__ __forceinline__ void write_rope(float2 *rope, size_t row, int pos, in
 }
 
 // ------------------------------------------------------------------------------- caller tree
-__global__ void tree_from_caller_kernel(TreeBufs t, const int32_t *__restrict__ tok,
-                                        const int32_t *__restrict__ parent,
-                                        const int32_t *__restrict__ n_nodes, int stride, int N,
+__global__ void tree_from_caller_kernel(TreeBufs t, const int32_t *tok,
+                                        const int32_t *parent,
+                                        const int32_t *n_nodes, int stride, int N,
                                         int *status) {
   pdl_launch_dependents();
   pdl_wait();
@@ -87,7 +87,7 @@ __global__ void tree_ancestors_kernel(TreeBufs t, int N) {
 }
 
 // ------------------------------------------------------------------------------- plans
-__global__ void plan_verify_kernel(TreeBufs t, PlanBufs p, const int32_t *__restrict__ seq_len,
+__global__ void plan_verify_kernel(TreeBufs t, PlanBufs p, const int32_t *seq_len,
                                    int N, int head_dim, float rope_base, int S_max, int *status) {
   pdl_launch_dependents();
   pdl_wait();
@@ -117,7 +117,7 @@ __global__ void plan_verify_kernel(TreeBufs t, PlanBufs p, const int32_t *__rest
 }
 
 // Draft pass 0 (EAGLE-style): the positions accepted last, as a chain on top of the head's cache.
-__global__ void plan_draft0_kernel(TreeBufs t, PlanBufs p, const int32_t *__restrict__ seq_len,
+__global__ void plan_draft0_kernel(TreeBufs t, PlanBufs p, const int32_t *seq_len,
                                    int N, int rows, int head_dim, float rope_base, int S_max,
                                    int *status) {
   pdl_launch_dependents();
@@ -165,7 +165,7 @@ __global__ void plan_medusa_kernel(TreeBufs t, PlanBufs p, int B, int N, int hea
 }
 
 // Draft pass p >= 1: the k frontier candidates of level p.
-__global__ void plan_draft_p_kernel(TreeBufs t, PlanBufs p, const int32_t *__restrict__ seq_len,
+__global__ void plan_draft_p_kernel(TreeBufs t, PlanBufs p, const int32_t *seq_len,
                                     int k, int pool, int pass, int head_dim, float rope_base,
                                     int S_max, int *status) {
   pdl_launch_dependents();
@@ -359,43 +359,65 @@ __global__ void expand_static_kernel(TreeBufs t, const int32_t *__restrict__ s_p
 }
 
 // ------------------------------------------------------------------------------- acceptance
-__global__ void accept_walk_kernel(TreeBufs t, const int32_t *__restrict__ tgt,
-                                   const float *__restrict__ hid,
-                                   const int32_t *__restrict__ forced_len, int32_t *seq_len,
+__global__ void accept_walk_kernel(TreeBufs t, const int32_t *tgt,
+                                   const float *hid,
+                                   const int32_t *forced_len, int32_t *seq_len,
                                    int32_t *out_tokens, int out_stride, int32_t *out_len, int N,
                                    int H) {
   __shared__ int s_path[128];
   __shared__ int s_len;
+  __shared__ int s_par[128], s_tok[128], s_tgt[128];
+  __shared__ int s_last;
   pdl_launch_dependents();
   pdl_wait();
   const int b = blockIdx.x;
-  if (threadIdx.x == 0) {
-    const int n = t.tree_n[b];
+  const int n = t.tree_n[b] < 128 ? t.tree_n[b] : 128;
+  for (int v = threadIdx.x; v < n; v += blockDim.x) {
+    s_par[v] = t.tree_parent[b * N + v];
+    s_tok[v] = t.tree_tok[b * N + v];
+    s_tgt[v] = tgt[b * N + v];
+  }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    // warp 0 walks down from the root; its lanes look at the children of the current node together
+    const int lane = threadIdx.x;
     const int f = forced_len ? forced_len[b] : 0;
     int u = 0, len = 1;
-    s_path[0] = 0;
+    if (lane == 0) s_path[0] = 0;
     while (true) {
       if (f > 0 && len >= f) break;
-      const int want = tgt[b * N + u];
-      int match = -1, first = -1;
-      for (int v = u + 1; v < n; ++v) {
-        if (t.tree_parent[b * N + v] != u) continue;
-        if (first < 0) first = v;
-        if (t.tree_tok[b * N + v] == want) { match = v; break; }
+      const int want = s_tgt[u];
+      int match = 0x7fffffff, first = 0x7fffffff;       // smallest matching child, smallest child
+      for (int v = u + 1 + lane; v < n; v += 32) {
+        if (s_par[v] != u) continue;
+        first = first < v ? first : v;
+        if (s_tok[v] == want) match = match < v ? match : v;
       }
-      int nxt = match;
-      if (nxt < 0 && f > 0) nxt = first;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const int m2 = __shfl_xor_sync(0xffffffffu, match, o), f2 = __shfl_xor_sync(0xffffffffu, first, o);
+        match = match < m2 ? match : m2;
+        first = first < f2 ? first : f2;
+      }
+      int nxt = match != 0x7fffffff ? match : -1;
+      if (nxt < 0 && f > 0 && first != 0x7fffffff) nxt = first;
       if (nxt < 0) break;
-      s_path[len++] = nxt;
+      if (lane == 0) s_path[len] = nxt;
+      ++len;
       u = nxt;
     }
-    const int bonus = tgt[b * N + u];
+    if (lane == 0) { s_len = len; s_last = u; }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int len = s_len, u = s_last;
+    const int bonus = s_tgt[u];
     const int S = seq_len[b];
     s_len = len;
     for (int i = 0; i < len; ++i) {
       t.acc_path[b * N + i] = s_path[i];
       if (i >= 1) {
-        const int tk = t.tree_tok[b * N + s_path[i]];
+        const int tk = s_tok[s_path[i]];
         t.pend_tok[b * N + i - 1] = tk;
         if (i - 1 < out_stride) out_tokens[(size_t)b * out_stride + i - 1] = tk;
       }
@@ -413,7 +435,12 @@ __global__ void accept_walk_kernel(TreeBufs t, const int32_t *__restrict__ tgt,
   for (int i = 0; i < len; ++i) {
     const float *src = hid + ((size_t)b * N + s_path[i]) * H;
     float *dst = t.pend_hid + ((size_t)b * N + i) * H;
-    for (int d = threadIdx.x; d < H; d += blockDim.x) dst[d] = src[d];
+    if ((H & 3) == 0) {
+      for (int d = threadIdx.x; d < (H >> 2); d += blockDim.x)
+        reinterpret_cast<float4 *>(dst)[d] = reinterpret_cast<const float4 *>(src)[d];
+    } else {
+      for (int d = threadIdx.x; d < H; d += blockDim.x) dst[d] = src[d];
+    }
   }
 }
 
