@@ -159,6 +159,8 @@ class KoalaOracle:
         n_draft_kv = K if cfg.head_kind == EAGLE else 0
         self.draft_k = [[np.zeros(shape, dtype) for _ in range(B)] for _ in range(n_draft_kv)]
         self.draft_v = [[np.zeros(shape, dtype) for _ in range(B)] for _ in range(n_draft_kv)]
+        self.alpha_hits = [0] * cfg.N      # [n-1]: iterations whose n-th draft token was accepted
+        self.alpha_trials = [0] * cfg.N    # [n-1]: iterations that offered an n-th draft token after n-1 accepted
         self.seq_len = [0] * B                  # tokens held by the target cache
         self.root_tok = [0] * B                 # x_S: the token the next tree is rooted at
         self.pend_hid: List[np.ndarray] = [np.zeros((0, cfg.H), dtype) for _ in range(B)]
@@ -412,6 +414,11 @@ class KoalaOracle:
             self.verify_tgt[b] = np.asarray([argmax_first(r) for r in logits], dtype=np.int64)
 
     # ------------------------------------------------------------------ accept + compaction
+    def reset_alpha(self):
+        """Clears the position-wise acceptance counters (they also count forced prompt chunks)."""
+        self.alpha_hits = [0] * self.cfg.N
+        self.alpha_trials = [0] * self.cfg.N
+
     def accept(self, forced_len: Optional[Sequence[int]] = None):
         """Greedy acceptance of the longest matching root path, then cache compaction.
 
@@ -448,6 +455,17 @@ class KoalaOracle:
                 path.append(nxt)
                 u = nxt
             ell = len(path)
+            # position-wise acceptance (the n-alpha metric of Section 4.1, metrics): the n-th draft
+            # token on the walked path was tried if the walk reached depth n-1 and that node has a
+            # child; it was hit if the walk went on to depth n
+            while len(self.alpha_hits) < ell:           # a caller's tree may be deeper than N
+                self.alpha_hits.append(0)
+                self.alpha_trials.append(0)
+            for n in range(1, ell):
+                self.alpha_hits[n - 1] += 1
+                self.alpha_trials[n - 1] += 1
+            if children[u]:
+                self.alpha_trials[ell - 1] += 1
             bonus = int(tgt[u])
             S = self.seq_len[b]
             for l in range(c.L):

@@ -160,3 +160,43 @@ def test_forced_length_rule_and_duplicate_siblings(hw):
     # duplicate sibling tokens: the lower-numbered child wins
     dup = [root, 20, 20, 30, 40, 50, 60]
     assert run(dup, [20, 5, 6, 0, 0, 0, 0], None) == ([20, 5], 2)
+
+
+def test_position_wise_acceptance_counts_on_planted_chains(hw, ar_stream):
+    """n-alpha (Section 4.1, metrics: accuracy of the n-th drafted token, chain drafts): a chain of
+    depth d whose first m tokens are the true continuation offers positions 1 .. min(m + 1, d)
+    and hits positions 1 .. m.  The expected counts are tallied here from (m, d) alone."""
+    first_root, truth = ar_stream
+    rng = np.random.default_rng(11)
+    o = KoalaOracle(CFG, hw)
+    o.prefill(prompts(CFG), 16)
+    o.reset_alpha()
+    hits, trials = [0] * CFG.N, [0] * CFG.N
+    emitted = 0
+    for _ in range(14):
+        d = int(rng.integers(1, 5))
+        m = int(rng.integers(0, d + 1))
+        tok = [o.root_tok[0]]
+        for i in range(d):
+            t = int(truth[emitted + i])
+            tok.append(t if i < m else (t + 1 + int(rng.integers(0, CFG.V - 1))) % CFG.V)
+        par = list(range(-1, d))
+        o.verify([(np.asarray(tok), np.asarray(par))])
+        _, lens = o.accept()
+        assert lens[0] == m + 1
+        emitted += lens[0]
+        for n in range(1, d + 1):
+            if n <= m + 1:
+                trials[n - 1] += 1
+            if n <= m:
+                hits[n - 1] += 1
+    assert o.alpha_hits == hits and o.alpha_trials == trials
+    assert all(h <= t for h, t in zip(hits, trials)) and trials[0] == 14
+    # a bushy tree counts the walked path only: the same tally with junk siblings around
+    o.reset_alpha()
+    tok, par = _planted_tree(rng, truth[emitted:], 2, 12, CFG.V)
+    tok[0] = o.root_tok[0]
+    o.verify([(np.asarray(tok), np.asarray(par))])
+    _, lens = o.accept()
+    assert lens[0] == 3 and o.alpha_hits[:3] == [1, 1, 0]
+    assert o.alpha_trials[:2] == [1, 1] and o.alpha_trials[2] in (0, 1)     # 1 iff the path's end has a (wrong) child
