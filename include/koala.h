@@ -187,6 +187,17 @@ int koala_verify(koala_ctx *ctx, const koala_tree *tree);
 int koala_accept(koala_ctx *ctx, const int32_t *forced_len, int32_t *out_tokens, int32_t out_stride,
                  int32_t *out_len);
 
+/* Position-wise acceptance counters, accumulated by every koala_accept since koala_init or the
+ * last reset (Section 4.1, metrics: the acceptance rate n-alpha, i.e. the accuracy on the n-th
+ * drafted token, which the paper measures with chain drafts).  Reading used here, for any tree:
+ * along the walked path, position n (n = 1 is the root's child) was offered if the walk reached
+ * depth n-1 and that node has a child, and hit if the walk went on to depth n; n-alpha =
+ * hits[n-1] / trials[n-1].  With chain trees this is the paper's metric.  Forced steps count as
+ * hits, so reset after ingesting a prompt.  hits / trials: HOST arrays of n_max <= 128 entries;
+ * the call copies on the context's stream and waits for it; reset != 0 clears the counters. */
+int koala_accept_stats(koala_ctx *ctx, uint64_t *hits, uint64_t *trials, int32_t n_max, int32_t reset);
+
+
 int koala_buffers(koala_ctx *ctx, koala_buffer_table *out);
 
 /* Run-time options.  KOALA_OPT_EXPAND_MODE splits koala_expand_tree for step-by-step checks:

@@ -90,6 +90,8 @@ def load_library(rebuild: bool = False) -> C.CDLL:
     lib.koala_expand_tree.argtypes = [C.c_void_p, C.c_int]
     lib.koala_verify.restype = C.c_int
     lib.koala_verify.argtypes = [C.c_void_p, C.POINTER(koala_tree)]
+    lib.koala_accept_stats.restype = C.c_int
+    lib.koala_accept_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32]
     lib.koala_accept.restype = C.c_int
     lib.koala_accept.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
     lib.koala_buffers.restype = C.c_int
@@ -262,6 +264,12 @@ class Koala:
         t = koala_tree(tok.data_ptr(), parent.data_ptr(), n_nodes.data_ptr(), tok.shape[1], int(n_max))
         self._keep = (tok, parent, n_nodes)
         self._check(self.lib.koala_verify(self._ctx, C.byref(t)))
+
+    def koala_accept_stats(self, n_max: int = 8, reset: bool = False):
+        """(hits, trials) of the position-wise acceptance counters as two lists of n_max integers."""
+        hits, trials = (C.c_uint64 * n_max)(), (C.c_uint64 * n_max)()
+        self._check(self.lib.koala_accept_stats(self._ctx, hits, trials, n_max, 1 if reset else 0))
+        return list(hits), list(trials)
 
     def koala_accept(self, forced_len: Optional[torch.Tensor] = None):
         """Returns (out_tokens [B, stride], out_len [B]) device tensors (asynchronous)."""

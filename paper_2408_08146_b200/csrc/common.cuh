@@ -196,6 +196,7 @@ struct TreeBufs {
   int32_t *topk_tok;
   float *topk_logp;
   int32_t *root_tok, *pend_tok, *n_pend, *acc_path, *acc_len, *acc_S;
+  unsigned long long *alpha_hits, *alpha_trials;   // [128] position-wise acceptance counters
   float *pend_hid;
 };
 struct PlanBufs {

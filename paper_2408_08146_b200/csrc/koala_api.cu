@@ -211,6 +211,8 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
   t.acc_path = w.take<int32_t>(M);
   t.acc_len = w.take<int32_t>(B);
   t.acc_S = w.take<int32_t>(B);
+  t.alpha_hits = w.take<unsigned long long>(128);
+  t.alpha_trials = w.take<unsigned long long>(128);
   t.pend_hid = w.take<float>((size_t)M * H);
   PlanBufs &p = c->p;
   p.pos = w.take<int32_t>(Mp);
@@ -505,6 +507,8 @@ int koala_init(const koala_config *cfg, const koala_weights *w, const koala_stat
   }
   // small state that must start at zero
   CU_TRY(cudaMemsetAsync(c->status, 0, 4 * sizeof(int), c->st));
+  CU_TRY(cudaMemsetAsync(c->t.alpha_hits, 0, 128 * sizeof(unsigned long long), c->st));
+  CU_TRY(cudaMemsetAsync(c->t.alpha_trials, 0, 128 * sizeof(unsigned long long), c->st));
   CU_TRY(cudaMemsetAsync(c->t.n_pend, 0, g.B * sizeof(int32_t), c->st));
   CU_TRY(cudaMemsetAsync(c->t.root_tok, 0, g.B * sizeof(int32_t), c->st));
   CU_TRY(cudaMemsetAsync(c->t.tree_n, 0, g.B * sizeof(int32_t), c->st));
@@ -617,6 +621,21 @@ int koala_accept(koala_ctx *c, const int32_t *forced_len, int32_t *out_tokens, i
   CU_TRY(kv_compact(LN(c), g.dtype, c->t, c->tk, c->tv, g.L, g.B, g.N, g.n_heads, g.head_dim, g.S_max));
   c->phase = PH_READY;
   c->last_pass = -1;
+  return KOALA_OK;
+}
+
+int koala_accept_stats(koala_ctx *c, uint64_t *hits, uint64_t *trials, int32_t n_max, int32_t reset) {
+  if (!c) return KOALA_E_INVALID;
+  if (n_max < 0 || n_max > 128 || (n_max > 0 && (!hits || !trials))) return fail(c, KOALA_E_INVALID, "bad n_max / null outputs");
+  if (n_max > 0) {
+    CU_TRY(cudaMemcpyAsync(hits, c->t.alpha_hits, (size_t)n_max * sizeof(uint64_t), cudaMemcpyDeviceToHost, c->st));
+    CU_TRY(cudaMemcpyAsync(trials, c->t.alpha_trials, (size_t)n_max * sizeof(uint64_t), cudaMemcpyDeviceToHost, c->st));
+  }
+  if (reset) {
+    CU_TRY(cudaMemsetAsync(c->t.alpha_hits, 0, 128 * sizeof(unsigned long long), c->st));
+    CU_TRY(cudaMemsetAsync(c->t.alpha_trials, 0, 128 * sizeof(unsigned long long), c->st));
+  }
+  CU_TRY(cudaStreamSynchronize(c->st));
   return KOALA_OK;
 }
 

@@ -407,6 +407,18 @@ __global__ void accept_walk_kernel(TreeBufs t, const int32_t *tgt,
       u = nxt;
     }
     if (lane == 0) { s_len = len; s_last = u; }
+    // position-wise acceptance (the n-alpha metric): position n was offered if the walk reached
+    // depth n-1 and that node has a child, and hit if the walk went on to depth n
+    int child = 0;
+    for (int v = u + 1 + lane; v < n; v += 32) child |= (s_par[v] == u);
+    child = __any_sync(0xffffffffu, child);
+    if (t.alpha_hits != nullptr) {
+      for (int i = 1 + lane; i < len && i <= 128; i += 32) {
+        atomicAdd(&t.alpha_hits[i - 1], 1ull);
+        atomicAdd(&t.alpha_trials[i - 1], 1ull);
+      }
+      if (lane == 0 && child && len <= 128) atomicAdd(&t.alpha_trials[len - 1], 1ull);
+    }
   }
   __syncthreads();
   if (threadIdx.x == 0) {

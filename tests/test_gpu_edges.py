@@ -10,6 +10,7 @@ import torch
 from oracle.koala_oracle import KoalaOracle, round_to_bf16
 from paper_2408_08146_b200 import Koala, KoalaError
 from tests.harness import kv_to_oracle, make_pair, tok_list
+from tests.helpers import HostWeights
 from tests.parity import assert_close, check_argmax
 from workloads import T7_EAGLE, TINY_EAGLE, reduced
 from workloads.generate import prompts, random_kv, uniform_ints
@@ -188,4 +189,50 @@ def test_call_order_and_argument_errors():
     with pytest.raises(KoalaError) as e:
         eng.koala_verify((tok, tok, torch.ones(1, dtype=torch.int32, device=DEV), 16))   # n_max > N
     assert e.value.code == 1
+    eng.close()
+
+
+def test_position_wise_acceptance_counters_match_the_oracle():
+    """n-alpha counters (Section 4.1, metrics): chains whose first m tokens are the target's own
+    greedy continuation, then free-running iterations with the head's real trees; the device
+    counters equal the oracle's and, for the planted part, the tally made here from (m, d)."""
+    cfg = TINY_EAGLE.with_(S_max=256)
+    eng, orc, store = make_pair(cfg)
+    pr = prompts(cfg)
+    eng.prefill(pr, 15)
+    orc.prefill(pr, 15)
+    truth_src = KoalaOracle(cfg, HostWeights(store, np.float64))
+    truth_src.prefill(pr, 64)
+    truth = truth_src.ar_greedy(80)[0]
+    eng.koala_accept_stats(1, reset=True)
+    orc.reset_alpha()
+    hits, trials = [0] * cfg.N, [0] * cfg.N
+    emitted = 0
+    for it in range(10):
+        d = 1 + (it * 3) % 5
+        m = (it * 7) % (d + 1)
+        tok = [int(orc.root_tok[0])]
+        for i in range(d):
+            t = int(truth[emitted + i])
+            tok.append(t if i < m else (t + 1 + 13 * it) % cfg.V)
+        par = list(range(-1, d))
+        eng.koala_verify(_tree_arrays(eng, [tok], [par]))
+        orc.verify([(np.asarray(tok), np.asarray(par))])
+        got = tok_list(*eng.koala_accept(None))
+        ref = orc.accept()
+        assert list(got[1]) == list(ref[1]) == [m + 1] and list(got[0][0]) == list(ref[0][0])
+        emitted += m + 1
+        for n in range(1, d + 1):
+            trials[n - 1] += n <= m + 1
+            hits[n - 1] += n <= m
+    g_hits, g_trials = eng.koala_accept_stats(cfg.N)
+    assert g_hits == hits == orc.alpha_hits[:cfg.N] and g_trials == trials == orc.alpha_trials[:cfg.N]
+    for _ in range(4):                                   # the head's own trees
+        got = tok_list(*eng.step())
+        ref = orc.step()
+        assert list(got[0]) == ref[0] and list(got[1]) == ref[1]
+    g_hits, g_trials = eng.koala_accept_stats(cfg.N, reset=True)
+    assert g_hits == orc.alpha_hits[:cfg.N] and g_trials == orc.alpha_trials[:cfg.N]
+    assert eng.koala_accept_stats(cfg.N) == ([0] * cfg.N, [0] * cfg.N)
+    assert eng.device_status() == 0
     eng.close()
