@@ -245,7 +245,9 @@ class KoalaOracle:
     def medusa_draft(self, h_last: np.ndarray):
         """Head i (0-based): x <- h_last; K times x <- x + SiLU(W_ij x + b_ij); logits = LM(x).
 
-        Non-autoregressive: all heads read the same hidden state; the LM head is shared.
+        Non-autoregressive: all heads read the same hidden state.  LM is the target's LM head,
+        shared by the heads, or - cfg.medusa_own_lm, Section 3.1's head as drawn: K x ResBlock
+        followed by a Linear of its own - the head's own [V, H] matrix "medusa.i.lm".
         Returns (logits [n_medusa_heads, V], features); head i ranks the token at tree level i+1.
         """
         c = self.cfg
@@ -256,6 +258,9 @@ class KoalaOracle:
                 x = x + silu(self.W(f"medusa.{i}.{j}.w") @ x + self.W(f"medusa.{i}.{j}.b"))
             feats.append(x)
         feats = np.stack(feats, axis=0)
+        if getattr(c, "medusa_own_lm", False):
+            logits = np.stack([self.W(f"medusa.{i}.lm") @ feats[i] for i in range(c.n_medusa_heads)], axis=0)
+            return logits, feats
         return feats @ self.W("lm_head").T, feats
 
     # ------------------------------------------------------------------ EAGLE-style draft pass

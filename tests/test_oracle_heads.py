@@ -244,3 +244,33 @@ def test_dynamic_selection_prunes_to_n_nodes_and_stays_ancestor_closed():
     _check_tree_invariants(o, cfg)
     vis = ancestor_matrix(o.tree_parent[0])
     assert vis[:, 0].all()
+
+
+def test_medusa_heads_with_their_own_linear():
+    """Section 3.1's Medusa head ends in a Linear per head.  Two pins that do not retype the
+    oracle's product: (1) with every head's matrix equal to the target's LM head the result is the
+    shared-head result; (2) with matrix i = the row pattern e_{(v + i) mod H} the logits are the
+    head's own features read off in that order."""
+    cfg = TINY_MEDUSA.with_(medusa_own_lm=True)
+    base = HostWeights(WeightStore(TINY_MEDUSA))
+    h = np.linspace(-1.0, 1.0, cfg.H)
+    shared_logits, feats = KoalaOracle(TINY_MEDUSA, base).medusa_draft(h)
+
+    class Same:
+        def __call__(self, name):
+            return base("lm_head") if name.endswith(".lm") else base(name)
+    same_logits, same_feats = KoalaOracle(cfg, Same()).medusa_draft(h)
+    assert np.array_equal(same_feats, feats)
+    np.testing.assert_allclose(same_logits, shared_logits, rtol=0, atol=1e-12)   # summation order only
+
+    class Pattern:
+        def __call__(self, name):
+            if name.endswith(".lm"):
+                i = int(name.split(".")[1])
+                w = np.zeros((cfg.V, cfg.H))
+                w[np.arange(cfg.V), (np.arange(cfg.V) + i) % cfg.H] = 1.0
+                return w
+            return base(name)
+    logits, f2 = KoalaOracle(cfg, Pattern()).medusa_draft(h)
+    for i in range(cfg.n_medusa_heads):
+        assert np.array_equal(logits[i], f2[i][(np.arange(cfg.V) + i) % cfg.H])

@@ -34,6 +34,7 @@ class KoalaConfig:
     B: int = 1            # sequences per step
     S_max: int = 256      # KV capacity per sequence
     n_medusa_heads: int = 0
+    medusa_own_lm: bool = False   # Medusa-style heads each end in a Linear of their own instead of the shared LM head
     rms_eps: float = 1e-5
     rope_base: float = 10000.0
     prompt_len: int = 64  # context length of the synthetic prompt (max, if ragged)

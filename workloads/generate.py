@@ -111,6 +111,8 @@ def weight_shapes(cfg: KoalaConfig) -> Dict[str, tuple]:
             for j in range(cfg.K):
                 shapes[f"medusa.{i}.{j}.w"] = (H, H)
                 shapes[f"medusa.{i}.{j}.b"] = (H,)
+            if cfg.medusa_own_lm:
+                shapes[f"medusa.{i}.lm"] = (V, H)
     return shapes
 
 
