@@ -94,6 +94,9 @@ typedef struct {
   const void *const *draft_layer_w; /* EAGLE: HOST array of K*9 device pointers */
   const void *const *res_w;         /* MEDUSA: HOST array of n_medusa_heads*K device pointers [H][H] */
   const void *const *res_b;         /* MEDUSA: same, [H] */
+  /* MEDUSA, optional: HOST array of n_medusa_heads device pointers [V][H], the Linear that ends
+   * each head in Section 3.1's drawing of the Medusa head.  NULL: every head uses lm_head. */
+  const void *const *medusa_lm;
   /* MEDUSA static topology, HOST arrays of N entries (node 0: parent -1, level 0) */
   const int32_t *static_parent, *static_level, *static_rank;
 } koala_weights;

@@ -42,7 +42,8 @@ class koala_weights(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
                 ("layer_w", C.POINTER(C.c_void_p)), ("fc_w", C.c_void_p), ("fc_b", C.c_void_p),
                 ("draft_layer_w", C.POINTER(C.c_void_p)), ("res_w", C.POINTER(C.c_void_p)),
-                ("res_b", C.POINTER(C.c_void_p)), ("static_parent", C.POINTER(C.c_int32)),
+                ("res_b", C.POINTER(C.c_void_p)), ("medusa_lm", C.POINTER(C.c_void_p)),
+                ("static_parent", C.POINTER(C.c_int32)),
                 ("static_level", C.POINTER(C.c_int32)), ("static_rank", C.POINTER(C.c_int32))]
 
 
@@ -223,6 +224,9 @@ class Koala:
             self._res_b = _ptr_array([weights[f"medusa.{i}.{j}.b"] for i, j in hk])
             w.res_w = C.cast(self._res_w, C.POINTER(C.c_void_p))
             w.res_b = C.cast(self._res_b, C.POINTER(C.c_void_p))
+            if getattr(cfg, "medusa_own_lm", False):
+                self._medusa_lm = _ptr_array([weights[f"medusa.{i}.lm"] for i in range(cfg.n_medusa_heads)])
+                w.medusa_lm = C.cast(self._medusa_lm, C.POINTER(C.c_void_p))
             if static_tree is None:
                 raise ValueError("Medusa-style heads need a static tree (parent, level, rank)")
             self._st = [_i32_array(a) for a in static_tree]

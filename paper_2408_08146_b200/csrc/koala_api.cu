@@ -49,7 +49,7 @@ struct koala_ctx {
   bool pdl, use_tc;
   const void *embed, *lm_head, *final_norm, *fc_w, *fc_b;
   std::vector<LayerW> layers, draft_layers;
-  std::vector<const void *> res_w, res_b;
+  std::vector<const void *> res_w, res_b, medusa_lm;
   void *tk, *tv, *dk, *dv;
   int32_t *seq_len;
   // derived sizes
@@ -414,8 +414,18 @@ int draft_medusa(koala_ctx *c) {
                           nullptr, xi, nullptr, B, H, g.rms_eps));
     }
   }
-  GemmMats lm{{c->lm_head, nullptr, nullptr}, {g.V, 0, 0}, 1};
-  K_TRY(do_gemm(c, c->xn, H, lm, R, c->draft_logits, g.V, nullptr));
+  if (c->medusa_lm.empty()) {
+    GemmMats lm{{c->lm_head, nullptr, nullptr}, {g.V, 0, 0}, 1};
+    K_TRY(do_gemm(c, c->xn, H, lm, R, c->draft_logits, g.V, nullptr));
+  } else {
+    // every head ends in its own Linear: one multiply per head over that head's B rows
+    for (int i = 0; i < nh; ++i) {
+      GemmMats lm{{c->medusa_lm[i], nullptr, nullptr}, {g.V, 0, 0}, 1};
+      const size_t off = (size_t)i * B * H * c->esz;
+      Operand xi{(unsigned char *)c->xn.hi + off, c->xn.lo ? (unsigned char *)c->xn.lo + off : nullptr};
+      K_TRY(do_gemm(c, xi, H, lm, B, c->draft_logits + (size_t)i * B * g.V, g.V, nullptr));
+    }
+  }
   c->draft_rows = R;
   return KOALA_OK;
 }
@@ -486,6 +496,11 @@ int koala_init(const koala_config *cfg, const koala_weights *w, const koala_stat
     const int n = g.n_medusa_heads * g.K;
     c->res_w.assign(w->res_w, w->res_w + n);
     c->res_b.assign(w->res_b, w->res_b + n);
+    if (w->medusa_lm) {
+      c->medusa_lm.assign(w->medusa_lm, w->medusa_lm + g.n_medusa_heads);
+      for (const void *p : c->medusa_lm)
+        if (!p) return fail(c, KOALA_E_INVALID, "null Medusa head matrix");
+    }
     for (int i = 0; i < n; ++i)
       if (!c->res_w[i] || !c->res_b[i]) return fail(c, KOALA_E_INVALID, "null Medusa block tensor");
     for (int u = 0; u < g.N; ++u) {

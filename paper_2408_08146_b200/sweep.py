@@ -1,13 +1,14 @@
 """Kernel-level sweep on the 7B shapes: draft latency against K, verify latency against tree size,
 context length and batch, each with its algorithmic bytes and the fraction of the HBM roofline.
 
-    python -m paper_2408_08146_b200.sweep [--what draft,verify] [--reps 10] [--json out.json]
+    python -m paper_2408_08146_b200.sweep [--what draft,verify,medusa] [--reps 10] [--json out.json]
 
 Run from the repository root (the seeded weight generator lives in `workloads/`).  Caches are
 zero-filled (the timing does not depend on their contents); lengths are set directly.
 The draft sweep runs whole iterations of an EAGLE-style head (D = 5 passes, top-10, 60-node tree,
 context 1024) on top of a one-layer target and times the draft / expand_tree calls only.
 The verify sweep times koala_verify on caller-supplied random trees.
+The medusa sweep times the Medusa-style draft with the shared LM head and with a Linear per head.
 """
 from __future__ import annotations
 
@@ -23,8 +24,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from workloads import T7_EAGLE  # noqa: E402
-from workloads.generate import WeightStore, uniform_ints  # noqa: E402
+from workloads import T7_EAGLE, T7_MEDUSA  # noqa: E402
+from workloads.generate import WeightStore, medusa_static_tree, uniform_ints  # noqa: E402
 
 from . import Koala  # noqa: E402
 
@@ -118,6 +119,47 @@ def draft_sweep(store, reps, peak):
     return rows
 
 
+def medusa_sweep(reps, peak):
+    """Medusa-style draft (4 heads x K = 2 residual blocks, one pass): the shared LM head against a
+    Linear of its own per head (Section 3.1's head as drawn), on a one-layer target."""
+    rows = []
+    for own in (False, True):
+        cfg = T7_MEDUSA.with_(L=1, medusa_own_lm=own, S_max=768)
+        store = WeightStore(cfg, DEV)
+        eng = Koala(cfg, store.tensors, static_tree=medusa_static_tree(cfg.N, cfg.n_medusa_heads, cfg.topk))
+        eng.seq_len.fill_(512)
+        bufs = eng.buffers()
+        bufs["n_pend"].fill_(3)
+        forced = torch.full((cfg.B,), 3, dtype=torch.int32, device=DEV)
+        stream = torch.cuda.current_stream()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        total, n = 0.0, 0
+        for it in range(3 + reps):
+            eng.seq_len.fill_(512)
+            e0.record(stream)
+            eng.koala_draft(0)
+            eng.koala_expand_tree(0)
+            e1.record(stream)
+            eng.koala_verify(None)
+            eng.koala_accept(forced)
+            torch.cuda.synchronize()
+            if it >= 3:
+                total += e0.elapsed_time(e1)
+                n += 1
+        assert eng.device_status() == 0
+        ms = total / n
+        nbytes = cfg.n_medusa_heads * cfg.K * cfg.H * cfg.H * 2 + (cfg.n_medusa_heads if own else 1) * cfg.V * cfg.H * 2
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        rows.append({"own_linear": own, "ms": round(ms, 4), "bytes": nbytes, "GBps": round(gbs, 1),
+                     "frac_measured": round(gbs / peak, 3)})
+        print(f"medusa draft, {'a Linear per head' if own else 'shared LM head   '}: {ms:6.3f} ms, {nbytes / 1e6:7.1f} MB, "
+              f"{gbs:6.0f} GB/s = {gbs / peak:.2f} of measured, {gbs / NOMINAL_GBS:.2f} of 8 TB/s", flush=True)
+        eng.close()
+        del eng, store
+        torch.cuda.empty_cache()
+    return rows
+
+
 def verify_sweep(store, reps, peak, tflops):
     rows = []
     grid = [(n, s, 1) for n in (16, 32, 64, 128) for s in (128, 512, 2048, 4096)]
@@ -157,8 +199,10 @@ def main():
     args = ap.parse_args()
     peak, tflops, src = measured_peak()
     print(f"HBM peak {peak:.0f} GB/s ({src}); nominal {NOMINAL_GBS:.0f} GB/s")
-    store = WeightStore(T7_EAGLE.with_(K=4), DEV)
     out = {"peak_GBps": peak, "peak_source": src}
+    if "medusa" in args.what:
+        out["medusa"] = medusa_sweep(args.reps, peak)
+    store = WeightStore(T7_EAGLE.with_(K=4), DEV) if ("draft" in args.what or "verify" in args.what) else None
     if "draft" in args.what:
         out["draft"] = draft_sweep(store, args.reps, peak)
     if "verify" in args.what:

@@ -166,6 +166,11 @@ def test_t7_medusa_full_size():
     _teacher_forced_iteration(T7_MEDUSA)
 
 
+def test_t7_medusa_heads_with_their_own_linear():
+    """Each head streams a [V][H] matrix of its own for its B rows (two target layers keep it short)."""
+    _teacher_forced_iteration(reduced(T7_MEDUSA, 2, medusa_own_lm=True))
+
+
 @pytest.mark.parametrize("K", [1, 2, 4])
 def test_t7_eagle_draft_and_verify(K):
     _teacher_forced_iteration(reduced(T7_EAGLE, 2, K=K))

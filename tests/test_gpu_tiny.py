@@ -107,6 +107,10 @@ def test_tiny_medusa_fp32():
     _run(TINY_MEDUSA.with_(S_max=192), 0, 6, 12)
 
 
+def test_tiny_medusa_heads_with_their_own_linear():
+    _run(TINY_MEDUSA.with_(S_max=192, medusa_own_lm=True, B=2, prompt_len=40, prompt_len_min=24, seed=6), 0, 5, 12)
+
+
 def test_tiny_eagle_batch_of_three_ragged_prompts():
     cfg = TINY_EAGLE.with_(B=3, prompt_len=48, prompt_len_min=20, S_max=160, seed=4)
     _run(cfg, 0, 4, 15)
