@@ -24,7 +24,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from workloads import T7_EAGLE, T7_MEDUSA  # noqa: E402
+from workloads import T33_EAGLE, T7_EAGLE, T7_MEDUSA  # noqa: E402
 from workloads.generate import WeightStore, medusa_static_tree, uniform_ints  # noqa: E402
 
 from . import Koala  # noqa: E402
@@ -72,11 +72,11 @@ def random_tree(cfg, n, seed):
     return to(tok), to(par), to(np.full(cfg.B, n, np.int32)), n
 
 
-def draft_sweep(store, reps, peak):
+def draft_sweep(store, reps, peak, base=T7_EAGLE, Ks=(1, 2, 3, 4)):
     rows = []
     S = 1024
-    for K in (1, 2, 3, 4):
-        cfg = T7_EAGLE.with_(L=1, K=K, S_max=S + 256, B=1)
+    for K in Ks:
+        cfg = base.with_(L=1, K=K, S_max=S + 256, B=1)
         eng = Koala(cfg, store.tensors)
         bufs = eng.buffers()
         eng.seq_len.fill_(S)
@@ -160,11 +160,12 @@ def medusa_sweep(reps, peak):
     return rows
 
 
-def verify_sweep(store, reps, peak, tflops):
+def verify_sweep(store, reps, peak, tflops, base=T7_EAGLE, grid=None):
     rows = []
-    grid = [(n, s, 1) for n in (16, 32, 64, 128) for s in (128, 512, 2048, 4096)]
-    grid += [(64, 512, b) for b in (2, 4, 8)] + [(64, 2048, b) for b in (2, 4, 8)]
-    base = T7_EAGLE.with_(K=1)
+    if grid is None:
+        grid = [(n, s, 1) for n in (16, 32, 64, 128) for s in (128, 512, 2048, 4096)]
+        grid += [(64, 512, b) for b in (2, 4, 8)] + [(64, 2048, b) for b in (2, 4, 8)]
+    base = base.with_(K=1)
     wbytes = base.L * layer_bytes(base) + base.V * base.H * 2
     for n, s, b in grid:
         cfg = base.with_(N=n, B=b, S_max=((s + n + 127) // 128) * 128, D=min(base.D, max(1, n - 1)))
@@ -196,12 +197,23 @@ def main():
     ap.add_argument("--what", default="draft,verify")
     ap.add_argument("--reps", type=int, default=10)
     ap.add_argument("--json", default="")
+    ap.add_argument("--model", default="7b", choices=["7b", "33b"],
+                    help="33b: the 33B shape (65 GB of weights): draft K = 1..8, verify at three points")
     args = ap.parse_args()
     peak, tflops, src = measured_peak()
     print(f"HBM peak {peak:.0f} GB/s ({src}); nominal {NOMINAL_GBS:.0f} GB/s")
     out = {"peak_GBps": peak, "peak_source": src}
     if "medusa" in args.what:
         out["medusa"] = medusa_sweep(args.reps, peak)
+    if args.model == "33b":
+        store = WeightStore(T33_EAGLE.with_(K=8), DEV)
+        if "draft" in args.what:
+            out["draft"] = draft_sweep(store, args.reps, peak, T33_EAGLE, (1, 2, 4, 6, 8))
+        if "verify" in args.what:
+            out["verify"] = verify_sweep(store, args.reps, peak, tflops, T33_EAGLE, [(16, 512, 1), (60, 512, 1), (60, 2048, 1)])
+        if args.json:
+            json.dump(out, open(args.json, "w"), indent=1)
+        return
     store = WeightStore(T7_EAGLE.with_(K=4), DEV) if ("draft" in args.what or "verify" in args.what) else None
     if "draft" in args.what:
         out["draft"] = draft_sweep(store, args.reps, peak)

@@ -10,7 +10,7 @@ import torch
 
 from tests.harness import kv_to_oracle, make_pair, tok_list
 from tests.parity import assert_close, check_argmax, check_topk
-from workloads import T13_EAGLE, T7_EAGLE, T7_MEDUSA, reduced
+from workloads import T13_EAGLE, T33_EAGLE, T7_EAGLE, T7_MEDUSA, reduced
 from workloads.generate import normal_tensor, prompt_lengths, random_kv, uniform_ints
 
 pytestmark = pytest.mark.gpu
@@ -182,3 +182,9 @@ def test_t7_eagle_cuda_core_path_agrees():
 
 def test_t13_eagle_batch4_ragged():
     _teacher_forced_iteration(reduced(T13_EAGLE, 2))
+
+
+@pytest.mark.parametrize("K", [2, 6])
+def test_t33_eagle_shape(K):
+    """33B-shaped layers (hidden 6656, 52 heads, FFN 17920) with a deeper head; one target layer."""
+    _teacher_forced_iteration(reduced(T33_EAGLE, 1, K=K, S_max=640, prompt_len=512))

@@ -74,6 +74,12 @@ T13_EAGLE = KoalaConfig(
     F=13824, V=32000, K=2, D=5, topk=10, N=64, B=4, S_max=2560, prompt_len=2048,
     prompt_len_min=512, seed=3)
 
+# 33B-shaped target (hidden 6656 = 52 heads x 128, FFN 17920, 60 layers), EAGLE-style head; the
+# paper expects larger K to pay off for larger targets (Section 4.2), so K is left to the caller.
+T33_EAGLE = KoalaConfig(
+    name="t33_eagle_bf16", dtype=BF16, head_kind=EAGLE, L=60, H=6656, n_heads=52, head_dim=128,
+    F=17920, V=32000, K=2, D=5, topk=10, N=60, B=1, S_max=1536, prompt_len=1024, seed=7)
+
 CONFIGS = [TINY_EAGLE, T7_MEDUSA, T7_EAGLE, T13_EAGLE]
 
 
