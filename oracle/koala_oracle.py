@@ -91,6 +91,32 @@ def top_k(values: np.ndarray, k: int) -> np.ndarray:
     return order[:k].astype(np.int64)
 
 
+def sample_index(w: np.ndarray, u: float) -> int:
+    """Inverse-CDF draw in index order from non-negative weights: the smallest j with
+    w_0 + .. + w_j > u * sum(w), u in [0, 1) (rounding can leave none: then the last j with w_j > 0)."""
+    c = np.cumsum(np.asarray(w, dtype=np.float64))
+    j = int(np.searchsorted(c, u * c[-1], side="right"))
+    if j >= len(c):
+        j = int(np.nonzero(np.asarray(w) > 0)[0][-1])
+    return j
+
+
+def speculative_sampling_step(d, q, drafted, u_accept, u_bonus):
+    """Acceptance of a chain of t drafted tokens by speculative sampling (Section 2.2, the
+    paragraph after Eq. 3).  d[i], q[i]: draft and target distributions at chain position i
+    (q has t + 1 rows); drafted[i] was drawn from d[i].  Token i is accepted with probability
+    min(1, q_i(x_i) / d_i(x_i)), i.e. iff u_accept[i] * d_i(x_i) < q_i(x_i); the first rejected
+    position f is redrawn from norm(max(0, q_f - d_f)) and the rest discarded; if all t are accepted
+    one more token is drawn from q_{t+1}.  Both draws use u_bonus.  Returns (accepted count, the
+    extra token)."""
+    t = len(drafted)
+    for i in range(t):
+        x = int(drafted[i])
+        if not (u_accept[i] * d[i][x] < q[i][x]):
+            return i, sample_index(np.maximum(0.0, np.asarray(q[i], np.float64) - np.asarray(d[i], np.float64)), u_bonus)
+    return t, sample_index(q[t], u_bonus)
+
+
 def round_to_bf16(x: np.ndarray) -> np.ndarray:
     """Round-to-nearest-even of float32 values to bfloat16 (8 significant bits), returned as float32.
 
@@ -159,6 +185,7 @@ class KoalaOracle:
         n_draft_kv = K if cfg.head_kind == EAGLE else 0
         self.draft_k = [[np.zeros(shape, dtype) for _ in range(B)] for _ in range(n_draft_kv)]
         self.draft_v = [[np.zeros(shape, dtype) for _ in range(B)] for _ in range(n_draft_kv)]
+        self.chain_d = [dict() for _ in range(cfg.B)]   # [b][level] draft distribution of a sampled chain
         self.alpha_hits = [0] * cfg.N      # [n-1]: iterations whose n-th draft token was accepted
         self.alpha_trials = [0] * cfg.N    # [n-1]: iterations that offered an n-th draft token after n-1 accepted
         self.seq_len = [0] * B                  # tokens held by the target cache
@@ -335,8 +362,13 @@ class KoalaOracle:
                 self.draft_feat[b], self.draft_logits[b] = f_hat, logits
 
     # ------------------------------------------------------------------ tree expansion
-    def expand_tree(self, p: int):
+    def expand_tree(self, p: int, u_draft=None):
         """Top-k expansion after draft pass p.
+
+        u_draft (one uniform per sequence, chain drafts only: k = 1): the level's token is drawn
+        from softmax(logits) by `sample_index` instead of being the arg-max (Section 2.2: the
+        draft distributions d_i govern the sampling of the drafted tokens); the distribution is
+        kept in chain_d[b][p] for `accept_sampled`.
 
         Dynamic tree (EAGLE-style): each row's k best tokens are taken from its logits (larger
         logit first, then smaller id); a candidate's score is its parent's score plus the token's
@@ -369,7 +401,13 @@ class KoalaOracle:
             parents = [-1] if p == 0 else list(self.frontier[b])
             for i, par in enumerate(parents):
                 base_score = self.dt(0.0) if par == -1 else pool[par]["score"]
-                for r, t in enumerate(top_k(logits[i], c.topk)):
+                picks = top_k(logits[i], c.topk)
+                if u_draft is not None:
+                    assert c.topk == 1, "drafted tokens are sampled on chains only"
+                    dist = np.exp(logp[i])
+                    self.chain_d[b][p] = dist
+                    picks = [sample_index(dist, float(u_draft[b]))]
+                for r, t in enumerate(picks):
                     pool.append({"level": p + 1, "parent": par, "rank": r, "tok": int(t),
                                  "score": self.dt(base_score + logp[i][t])})
             new_ids = list(range(first_new, len(pool)))
@@ -419,6 +457,35 @@ class KoalaOracle:
             self.verify_tgt[b] = np.asarray([argmax_first(r) for r in logits], dtype=np.int64)
 
     # ------------------------------------------------------------------ accept + compaction
+    def _commit_path(self, b: int, path, bonus: int, last_has_child: bool):
+        """Bookkeeping shared by the acceptance rules: counters, cache compaction, pending rows."""
+        c = self.cfg
+        tok = self.tree_tok[b]
+        ell = len(path)
+        # position-wise acceptance (the n-alpha metric of Section 4.1, metrics): the n-th draft
+        # token on the walked path was tried if the walk reached depth n-1 and that node has a
+        # child; it was hit if the walk went on to depth n
+        while len(self.alpha_hits) < ell:           # a caller's tree may be deeper than N
+            self.alpha_hits.append(0)
+            self.alpha_trials.append(0)
+        for n in range(1, ell):
+            self.alpha_hits[n - 1] += 1
+            self.alpha_trials[n - 1] += 1
+        if last_has_child:
+            self.alpha_trials[ell - 1] += 1
+        S = self.seq_len[b]
+        for l in range(c.L):
+            for cache in (self.target_k[l][b], self.target_v[l][b]):
+                fresh = np.zeros_like(cache)
+                fresh[:S] = cache[:S]
+                fresh[S:S + ell] = cache[S + np.asarray(path)]
+                cache[...] = fresh
+        self.pend_hid[b] = self.verify_hid[b][np.asarray(path)].copy()
+        self.pend_tok[b] = [int(tok[v]) for v in path[1:]]
+        self.seq_len[b] = S + ell
+        self.root_tok[b] = bonus
+        return [int(tok[v]) for v in path[1:]] + [bonus], ell
+
     def reset_alpha(self):
         """Clears the position-wise acceptance counters (they also count forced prompt chunks)."""
         self.alpha_hits = [0] * self.cfg.N
@@ -459,31 +526,27 @@ class KoalaOracle:
                     break
                 path.append(nxt)
                 u = nxt
-            ell = len(path)
-            # position-wise acceptance (the n-alpha metric of Section 4.1, metrics): the n-th draft
-            # token on the walked path was tried if the walk reached depth n-1 and that node has a
-            # child; it was hit if the walk went on to depth n
-            while len(self.alpha_hits) < ell:           # a caller's tree may be deeper than N
-                self.alpha_hits.append(0)
-                self.alpha_trials.append(0)
-            for n in range(1, ell):
-                self.alpha_hits[n - 1] += 1
-                self.alpha_trials[n - 1] += 1
-            if children[u]:
-                self.alpha_trials[ell - 1] += 1
-            bonus = int(tgt[u])
-            S = self.seq_len[b]
-            for l in range(c.L):
-                for cache in (self.target_k[l][b], self.target_v[l][b]):
-                    fresh = np.zeros_like(cache)
-                    fresh[:S] = cache[:S]
-                    fresh[S:S + ell] = cache[S + np.asarray(path)]
-                    cache[...] = fresh
-            self.pend_hid[b] = self.verify_hid[b][np.asarray(path)].copy()
-            self.pend_tok[b] = [int(tok[v]) for v in path[1:]]
-            self.seq_len[b] = S + ell
-            self.root_tok[b] = bonus
-            out_tok.append([int(tok[v]) for v in path[1:]] + [bonus])
+            toks_b, ell = self._commit_path(b, path, int(tgt[u]), bool(children[u]))
+            out_tok.append(toks_b)
+            out_len.append(ell)
+        return out_tok, out_len
+
+    def accept_sampled(self, u_accept, u_bonus):
+        """Speculative-sampling acceptance of a chain tree (Section 2.2; temperature 1): position i
+        of the chain is judged with q_i = softmax of the target's logits at node i-1 and the draft
+        distribution kept by `expand_tree(p, u_draft)`; see `speculative_sampling_step`.
+        u_accept[b][i], u_bonus[b]: uniforms in [0, 1).  Returns (tokens, lengths) like `accept`."""
+        c = self.cfg
+        out_tok, out_len = [], []
+        for b in range(c.B):
+            tok, parent = self.tree_tok[b], self.tree_parent[b]
+            n = len(tok)
+            assert all(int(parent[i]) == i - 1 for i in range(n)), "speculative sampling is defined on chains"
+            q = np.exp(log_softmax(self.verify_logits[b][:n]))
+            d = [self.chain_d[b][i] for i in range(n - 1)]
+            a, bonus = speculative_sampling_step(d, q, [int(t) for t in tok[1:]], u_accept[b], float(u_bonus[b]))
+            toks_b, ell = self._commit_path(b, list(range(a + 1)), int(bonus), a + 1 < n)
+            out_tok.append(toks_b)
             out_len.append(ell)
         return out_tok, out_len
 
