@@ -190,6 +190,28 @@ int koala_verify(koala_ctx *ctx, const koala_tree *tree);
 int koala_accept(koala_ctx *ctx, const int32_t *forced_len, int32_t *out_tokens, int32_t out_stride,
                  int32_t *out_len);
 
+/* Speculative sampling on chain drafts (Section 2.2, the paragraph after Eq. 3; the paper's
+ * non-greedy runs use temperature 1).  Only for an EAGLE-style head with topk = 1, i.e. a chain of
+ * D drafted tokens; the paper gives no rule for a tree.  All random numbers are the caller's.
+ *
+ * koala_set_sampling(ctx, u_draft): while u_draft (DEVICE [B][D], uniforms in [0, 1)) is non-null,
+ * koala_expand_tree(p) draws sequence b's level-(p+1) token from d = softmax(draft logits) with
+ * u_draft[b][p] (inverse CDF in token-id order: the smallest id whose cumulative probability
+ * exceeds u) instead of taking the arg-max, and keeps d.  NULL switches back to greedy drafts.
+ * The array is read when the kernels run: keep it alive and unchanged until then.
+ *
+ * koala_accept_sampled replaces koala_accept after koala_verify(ctx, NULL) of such a chain: with
+ * q_i = softmax of the target's logits at chain node i-1, drafted token i is accepted iff
+ * u_accept[b][i-1] * d_i(x_i) < q_i(x_i) (probability min(1, q_i/d_i)); the first rejected
+ * position is redrawn from max(0, q_f - d_f) normalised, later tokens are dropped; if all D are
+ * accepted one more token is drawn from q_{D+1}.  Both draws use u_bonus[b] and the same inverse
+ * CDF.  u_accept: DEVICE [B][D]; u_bonus: DEVICE [B].  Outputs, cache compaction, counters and the
+ * next root as in koala_accept (the extra token takes the place of the bonus token).  A tree that
+ * is not a chain sets the device status to KOALA_E_INVALID. */
+int koala_set_sampling(koala_ctx *ctx, const float *u_draft);
+int koala_accept_sampled(koala_ctx *ctx, const float *u_accept, const float *u_bonus, int32_t *out_tokens,
+                         int32_t out_stride, int32_t *out_len);
+
 /* Position-wise acceptance counters, accumulated by every koala_accept since koala_init or the
  * last reset (Section 4.1, metrics: the acceptance rate n-alpha, i.e. the accuracy on the n-th
  * drafted token, which the paper measures with chain drafts).  Reading used here, for any tree:

@@ -91,6 +91,10 @@ def load_library(rebuild: bool = False) -> C.CDLL:
     lib.koala_expand_tree.argtypes = [C.c_void_p, C.c_int]
     lib.koala_verify.restype = C.c_int
     lib.koala_verify.argtypes = [C.c_void_p, C.POINTER(koala_tree)]
+    lib.koala_set_sampling.restype = C.c_int
+    lib.koala_set_sampling.argtypes = [C.c_void_p, C.c_void_p]
+    lib.koala_accept_sampled.restype = C.c_int
+    lib.koala_accept_sampled.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
     lib.koala_accept_stats.restype = C.c_int
     lib.koala_accept_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32]
     lib.koala_accept.restype = C.c_int
@@ -268,6 +272,17 @@ class Koala:
         t = koala_tree(tok.data_ptr(), parent.data_ptr(), n_nodes.data_ptr(), tok.shape[1], int(n_max))
         self._keep = (tok, parent, n_nodes)
         self._check(self.lib.koala_verify(self._ctx, C.byref(t)))
+
+    def koala_set_sampling(self, u_draft: Optional[torch.Tensor]):
+        """u_draft: float32 device tensor [B][D] of uniforms (kept alive by the caller), or None."""
+        self._u_draft = u_draft
+        self._check(self.lib.koala_set_sampling(self._ctx, u_draft.data_ptr() if u_draft is not None else None))
+
+    def koala_accept_sampled(self, u_accept: torch.Tensor, u_bonus: torch.Tensor):
+        self._check(self.lib.koala_accept_sampled(self._ctx, u_accept.data_ptr(), u_bonus.data_ptr(),
+                                                  self.out_tokens.data_ptr(), self.out_stride,
+                                                  self.out_len.data_ptr()))
+        return self.out_tokens, self.out_len
 
     def koala_accept_stats(self, n_max: int = 8, reset: bool = False):
         """(hits, trials) of the position-wise acceptance counters as two lists of n_max integers."""

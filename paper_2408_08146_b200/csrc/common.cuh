@@ -223,4 +223,12 @@ cudaError_t accept_walk(Launch L, TreeBufs t, const int32_t *verify_tgt, const f
 cudaError_t kv_compact(Launch L, int dtype, TreeBufs t, void *k_cache, void *v_cache, int L_layers,
                        int B, int N, int n_heads, int head_dim, int S_max);
 
+// sampling.cu : speculative sampling on chain drafts (one row / one chain per sequence)
+cudaError_t sample_rows(Launch L, const float *logits, const float *u, int u_stride, int u_off, int32_t *tok,
+                        float *logp, float *probs, int R, int V);
+cudaError_t accept_sampled(Launch L, TreeBufs t, const float *verify_logits, const float *verify_hid,
+                           const float *chain_d, const float *u_accept, const float *u_bonus, int32_t *seq_len,
+                           int32_t *out_tokens, int out_stride, int32_t *out_len, int B, int N, int H, int V, int D,
+                           int *status);
+
 }  // namespace koala

@@ -63,6 +63,8 @@ struct koala_ctx {
   float *x, *qbuf, *P, *verify_logits, *draft_logits, *verify_hid, *feat[2], *mx;
   Operand xn, attn_out, act, cat, lmin;
   Operand qpair;           // rotated queries as a bf16 pair (bf16 configurations)
+  float *chain_d;          // [B][D][V] draft distributions of a sampled chain (k = 1 configurations)
+  const float *u_draft;    // device [B][D] uniforms: drafted tokens are sampled while non-null
   bool pair;              // bf16 activations kept as hi + lo
   int32_t *verify_tgt, *s_parent, *s_level, *s_rank;
   int *status;
@@ -211,6 +213,7 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
   t.acc_path = w.take<int32_t>(M);
   t.acc_len = w.take<int32_t>(B);
   t.acc_S = w.take<int32_t>(B);
+  c->chain_d = (cfg.head_kind == KOALA_EAGLE && k == 1) ? w.take<float>((size_t)B * cfg.D * V) : nullptr;
   t.alpha_hits = w.take<unsigned long long>(128);
   t.alpha_trials = w.take<unsigned long long>(128);
   t.pend_hid = w.take<float>((size_t)M * H);
@@ -455,6 +458,7 @@ int koala_init(const koala_config *cfg, const koala_weights *w, const koala_stat
   c->poll_ev = nullptr;
   c->poll_pending = false;
   c->last_status = 0;
+  c->u_draft = nullptr;
   char why[128];
   if (!config_ok(cfg, why, sizeof(why))) return fail(c, KOALA_E_INVALID, "%s", why);
   if (!w || !st) return fail(c, KOALA_E_INVALID, "null weights or state");
@@ -575,8 +579,15 @@ int koala_expand_tree(koala_ctx *c, int pass) {
   const koala_config &g = c->cfg;
   if (c->phase != PH_DRAFTED || c->last_pass != pass)
     return fail(c, KOALA_E_STATE, "koala_expand_tree(%d) must follow koala_draft(%d)", pass, pass);
-  if (c->expand_mode != 2)
-    CU_TRY(topk_logp(LN(c), c->draft_logits, c->t.topk_tok, c->t.topk_logp, c->draft_rows, g.V, g.topk));
+  if (c->expand_mode != 2) {
+    if (c->u_draft != nullptr && c->draft_rows == g.B) {
+      // chain drafts with sampled tokens: token ~ softmax(logits), the distribution is kept
+      CU_TRY(sample_rows(LN(c), c->draft_logits, c->u_draft, g.D, pass, c->t.topk_tok, c->t.topk_logp, c->chain_d,
+                         g.B, g.V));
+    } else {
+      CU_TRY(topk_logp(LN(c), c->draft_logits, c->t.topk_tok, c->t.topk_logp, c->draft_rows, g.V, g.topk));
+    }
+  }
   if (c->expand_mode == 1) return KOALA_OK;
   if (g.head_kind == KOALA_MEDUSA) {
     CU_TRY(expand_static(LN(c), c->t, c->s_parent, c->s_level, c->s_rank, g.B, g.N, g.topk));
@@ -633,6 +644,31 @@ int koala_accept(koala_ctx *c, const int32_t *forced_len, int32_t *out_tokens, i
   if (c->phase != PH_VERIFIED) return fail(c, KOALA_E_STATE, "koala_accept must follow koala_verify");
   CU_TRY(accept_walk(LN(c), c->t, c->verify_tgt, c->verify_hid, forced_len, c->seq_len, out_tokens,
                      out_stride, out_len, g.B, g.N, g.H));
+  CU_TRY(kv_compact(LN(c), g.dtype, c->t, c->tk, c->tv, g.L, g.B, g.N, g.n_heads, g.head_dim, g.S_max));
+  c->phase = PH_READY;
+  c->last_pass = -1;
+  return KOALA_OK;
+}
+
+int koala_set_sampling(koala_ctx *c, const float *u_draft) {
+  if (!c) return KOALA_E_INVALID;
+  if (u_draft != nullptr && c->chain_d == nullptr)
+    return fail(c, KOALA_E_INVALID, "sampled drafts need an EAGLE-style head with topk = 1 (chain drafts)");
+  c->u_draft = u_draft;
+  return KOALA_OK;
+}
+
+int koala_accept_sampled(koala_ctx *c, const float *u_accept, const float *u_bonus, int32_t *out_tokens,
+                         int32_t out_stride, int32_t *out_len) {
+  if (!c) return KOALA_E_INVALID;
+  const koala_config &g = c->cfg;
+  if (!u_accept || !u_bonus || !out_tokens || !out_len || out_stride < 1) return fail(c, KOALA_E_INVALID, "null arguments");
+  if (c->chain_d == nullptr || c->u_draft == nullptr)
+    return fail(c, KOALA_E_STATE, "koala_accept_sampled needs sampled chain drafts (koala_set_sampling)");
+  if (c->phase != PH_VERIFIED || c->last_tree_from_caller)
+    return fail(c, KOALA_E_STATE, "koala_accept_sampled must follow koala_verify of the drafted chain");
+  CU_TRY(accept_sampled(LN(c), c->t, c->verify_logits, c->verify_hid, c->chain_d, u_accept, u_bonus, c->seq_len,
+                        out_tokens, out_stride, out_len, g.B, g.N, g.H, g.V, g.D, c->status));
   CU_TRY(kv_compact(LN(c), g.dtype, c->t, c->tk, c->tv, g.L, g.B, g.N, g.n_heads, g.head_dim, g.S_max));
   c->phase = PH_READY;
   c->last_pass = -1;
