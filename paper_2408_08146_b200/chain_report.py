@@ -1,6 +1,6 @@
 """The paper's three metrics (Section 4.1) from the library's own counters, with chain drafts.
 
-    python -m paper_2408_08146_b200.chain_report [--layers 32] [--K 1] [--depth 3] [--iters 40]
+    python -m paper_2408_08146_b200.chain_report [--layers 32] [--K 1] [--depth 3] [--iters 40] [--sampled]
 
 Runs an EAGLE-style head on the 7B shape in chain mode (top-1 per level, a tree of depth+1 nodes,
 no tree attention needed), free-running with greedy acceptance, and prints
@@ -29,14 +29,27 @@ from workloads.generate import WeightStore, prompts  # noqa: E402
 from . import Koala  # noqa: E402
 
 
-def timed_steps(eng, n):
+def sampled_step(eng, cfg, u):
+    """One iteration with sampled drafts and speculative-sampling acceptance (Section 2.2)."""
+    eng.koala_set_sampling(u[0])
+    for p in range(cfg.D):
+        eng.koala_draft(p)
+        eng.koala_expand_tree(p)
+    eng.koala_verify(None)
+    return eng.koala_accept_sampled(u[1], u[2])
+
+
+def timed_steps(eng, n, cfg=None, uniforms=None):
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     total = 0
     e0.record()
     lens = []
-    for _ in range(n):
-        lens.append(eng.step()[1])
+    for i in range(n):
+        if uniforms is not None:
+            lens.append(sampled_step(eng, cfg, uniforms[i])[1].clone())
+        else:
+            lens.append(eng.step()[1].clone())
     e1.record()
     torch.cuda.synchronize()
     for ln in lens:
@@ -51,6 +64,8 @@ def main():
     ap.add_argument("--depth", type=int, default=3)
     ap.add_argument("--iters", type=int, default=40)
     ap.add_argument("--context", type=int, default=256)
+    ap.add_argument("--sampled", action="store_true",
+                    help="sampled drafts + speculative-sampling acceptance (temperature 1) instead of greedy")
     args = ap.parse_args()
     d = args.depth
     need = args.context + (args.iters + 8) * (d + 1) + 64
@@ -59,10 +74,15 @@ def main():
     store = WeightStore(chain, "cuda:0")
     eng = Koala(chain, store.tensors)
     eng.prefill(prompts(chain), chain.N)
-    for _ in range(3):
-        eng.step()
+    uniforms = None
+    if args.sampled:
+        g = torch.Generator(device="cuda:0").manual_seed(1)
+        uniforms = [(torch.rand(1, d, device="cuda:0", generator=g), torch.rand(1, d, device="cuda:0", generator=g),
+                     torch.rand(1, device="cuda:0", generator=g)) for _ in range(args.iters + 3)]
+    for i in range(3):
+        sampled_step(eng, chain, uniforms[args.iters + i]) if args.sampled else eng.step()
     eng.koala_accept_stats(1, reset=True)
-    ms, toks = timed_steps(eng, args.iters)
+    ms, toks = timed_steps(eng, args.iters, chain, uniforms)
     hits, trials = eng.koala_accept_stats(d)
     assert eng.device_status() == 0
     eng.close()
@@ -94,6 +114,7 @@ def main():
     eng.close()
     ell = toks / args.iters
     spec_ms_per_tok = ms / max(1, toks)
+    print("sampled drafts, speculative-sampling acceptance" if args.sampled else "greedy drafts, greedy acceptance")
     print(f"chain drafts, depth {d}, K = {args.K}, {args.layers} layers, context {args.context}, {args.iters} iterations")
     print(f"  average acceptance length l = {ell:.3f} tokens per target forward")
     for n in range(1, d + 1):
