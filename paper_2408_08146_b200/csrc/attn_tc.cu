@@ -61,6 +61,20 @@ __device__ __forceinline__ void split_pack(float x, float y, uint32_t &hi, uint3
   hi = *reinterpret_cast<const uint32_t *>(&h);
   lo = *reinterpret_cast<const uint32_t *>(&l);
 }
+// 2^x for x <= 0 (or -inf): one MUFU instruction; results below 2^-126 flush to zero
+__device__ __forceinline__ float ex2_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Probabilities p in [0, 1] as a bf16 pair: hi = p truncated to bf16 (exactly representable, so
+// p - hi is exact), lo = that remainder rounded to bf16.  |p - hi - lo| <= 2^-17 p.
+__device__ __forceinline__ void split_pack_trunc(float x, float y, uint32_t &hi, uint32_t &lo) {
+  const uint32_t xb = __float_as_uint(x) & 0xffff0000u, yb = __float_as_uint(y) & 0xffff0000u;
+  hi = __byte_perm(xb, yb, 0x7632);                 // (y.hi16 << 16) | x.hi16
+  const __nv_bfloat162 l = __floats2bfloat162_rn(x - __uint_as_float(xb), y - __uint_as_float(yb));
+  lo = *reinterpret_cast<const uint32_t *>(&l);
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -347,10 +361,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         uint32_t hi[4], lo[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const float p0 = exp2f(__uint_as_float(v[ch * 8 + 2 * e]) - mu);
-          const float p1 = exp2f(__uint_as_float(v[ch * 8 + 2 * e + 1]) - mu);
+          const float p0 = ex2_fast(__uint_as_float(v[ch * 8 + 2 * e]) - mu);
+          const float p1 = ex2_fast(__uint_as_float(v[ch * 8 + 2 * e + 1]) - mu);
           l_t += p0 + p1;
-          split_pack(p0, p1, hi[e], lo[e]);
+          split_pack_trunc(p0, p1, hi[e], lo[e]);
         }
         const uint32_t off = (((uint32_t)(ch + (NC / 8) * half)) ^ psw) << 4;
         st_shared_v4(pb + off, hi[0], hi[1], hi[2], hi[3]);
