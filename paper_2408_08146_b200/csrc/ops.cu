@@ -635,6 +635,121 @@ topk_logp_fast_kernel(const float *logits, int32_t *__restrict__ tok, float *__r
   }
 }
 
+// The same result on eight CTAs per row (a thread-block cluster): CTA p takes an eighth of the
+// row - 16 strided elements per thread in registers - and extracts its k best (every warp the k
+// best of its 512 elements with shuffles, warp 0 the k best of those 8 * k) together with its
+// (max, sum of exponentials); after a cluster barrier CTA 0 reads the eight candidate lists and
+// the eight (max, sum) pairs through distributed shared memory, takes the k best of the 8 * k
+// candidates (ties still go to the smaller id) and forms the log-sum-exp.  V <= 32768, k <= 32.
+constexpr int TKP = 8;            // CTAs per row
+__global__ void __launch_bounds__(256)
+topk_logp_cluster_kernel(const float *logits, int32_t *__restrict__ tok, float *__restrict__ logp, int V, int k) {
+  __shared__ ValIdx cand[8 * 32];
+  __shared__ ValIdx mine[32];     // this CTA's k best, read by CTA 0
+  __shared__ float s_ms[2];       // this CTA's (max, sum of exp(v - max))
+  __shared__ float redf[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int part = blockIdx.x, r = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+  const int chunk = (((V + TKP - 1) / TKP) + 255) & ~255;          // ids per CTA, a multiple of 256
+  const int base = part * chunk;
+  const float *row = logits + (size_t)r * V;
+  float vals[16];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const int i = base + tid + 256 * j;
+    vals[j] = (tid + 256 * j < chunk && i < V) ? row[i] : -INFINITY;
+    mx = fmaxf(mx, vals[j]);
+  }
+  mx = warp_max(mx);
+  if (lane == 0) redf[w] = mx;
+  __syncthreads();
+  mx = warp_max(lane < 8 ? redf[lane] : -INFINITY);
+  __syncthreads();
+  float se = 0.f;
+  if (mx != -INFINITY) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) se += expf(vals[j] - mx);
+  }
+  se = warp_sum(se);
+  if (lane == 0) redf[w] = se;
+  __syncthreads();
+  se = warp_sum(lane < 8 ? redf[lane] : 0.f);
+  if (tid == 0) { s_ms[0] = mx; s_ms[1] = se; }
+  for (int rnd = 0; rnd < k; ++rnd) {
+    ValIdx best{-INFINITY, 0x7fffffff};
+#pragma unroll
+    for (int j = 0; j < 16; ++j) best = better(best, ValIdx{vals[j], vals[j] == -INFINITY ? 0x7fffffff : base + tid + 256 * j});
+    best = warp_argmax(best);
+    if (best.i != 0x7fffffff && ((best.i - base) & 255) == tid) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (j == ((best.i - base) >> 8)) vals[j] = -INFINITY;
+    }
+    if (lane == 0) cand[w * k + rnd] = best;
+  }
+  __syncthreads();
+  if (w == 0) {
+    const int n = 8 * k;
+    for (int rnd = 0; rnd < k; ++rnd) {
+      ValIdx best{-INFINITY, 0x7fffffff};
+      int at = -1;
+      for (int c = lane; c < n; c += 32) {
+        const ValIdx x = cand[c];
+        if (x.v > best.v || (x.v == best.v && x.i < best.i)) { best = x; at = c; }
+      }
+      const ValIdx win = warp_argmax(best);
+      if (at >= 0 && best.i == win.i && win.i != 0x7fffffff) cand[at] = ValIdx{-INFINITY, 0x7fffffff};
+      __syncwarp();
+      if (lane == 0) mine[rnd] = win;
+    }
+  }
+  __syncthreads();
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+  if (part == 0 && w == 0) {
+    // lane l holds candidate l of every CTA (eight registers) and CTA (l % 8)'s (max, sum)
+    const uint32_t a_mine = (uint32_t)__cvta_generic_to_shared(&mine[lane < k ? lane : 0]);
+    const uint32_t a_ms = (uint32_t)__cvta_generic_to_shared(&s_ms[0]);
+    ValIdx c8[TKP];
+#pragma unroll
+    for (int j = 0; j < TKP; ++j) {
+      uint32_t ra;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a_mine), "r"(j));
+      float v; int id;
+      asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+      asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(id) : "r"(ra + 4) : "memory");
+      c8[j] = lane < k ? ValIdx{v, id} : ValIdx{-INFINITY, 0x7fffffff};
+    }
+    uint32_t rb;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rb) : "r"(a_ms), "r"(lane & 7));
+    float mj, sj;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(mj) : "r"(rb) : "memory");
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(sj) : "r"(rb + 4) : "memory");
+    const float M = warp_max(mj);
+    float part_sum = (lane < 8 && mj != -INFINITY) ? sj * expf(mj - M) : 0.f;
+    const float lse = M + logf(warp_sum(part_sum));
+    for (int rnd = 0; rnd < k; ++rnd) {
+      ValIdx best{-INFINITY, 0x7fffffff};
+#pragma unroll
+      for (int j = 0; j < TKP; ++j) best = better(best, c8[j]);
+      const ValIdx win = warp_argmax(best);
+#pragma unroll
+      for (int j = 0; j < TKP; ++j)
+        if (c8[j].i == win.i) c8[j] = ValIdx{-INFINITY, 0x7fffffff};
+      if (lane == 0) {
+        tok[(size_t)r * k + rnd] = win.i;
+        logp[(size_t)r * k + rnd] = win.v - lse;
+      }
+    }
+  }
+  // no CTA leaves while CTA 0 may still read its shared memory
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+
 }  // namespace
 
 #define DISPATCH_T(dtype, ...)                \
@@ -746,6 +861,23 @@ cudaError_t argmax_rows(Launch L, const float *logits, int32_t *out, int R, int 
 }
 
 cudaError_t topk_logp(Launch L, const float *logits, int32_t *tok, float *logp, int R, int V, int k) {
+  if (V <= 32768 && k <= 32 && V >= 4096) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(TKP, R);
+    cfg.blockDim = dim3(256);
+    cfg.stream = L.st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = L.pdl ? 1 : 0;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = TKP;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    ++g_launches;
+    return cudaLaunchKernelEx(&cfg, topk_logp_cluster_kernel, logits, tok, logp, V, k);
+  }
   if (V <= 32768 && k <= 32)
     return launch_k(topk_logp_fast_kernel, dim3(R), dim3(1024), 0, L.st, L.pdl, logits, tok, logp, V, k);
   const size_t smem = (size_t)V * sizeof(float);
