@@ -249,6 +249,27 @@ __global__ void eagle_concat_kernel(const float *feat_src,
   }
 }
 
+// The same with four elements per thread and the row spread over grid.y CTAs (H % 4 == 0): one
+// trip to memory per thread instead of a loop of dependent ones.
+template <typename T>
+__global__ void eagle_concat_vec_kernel(const float *feat_src, const int32_t *row_src, const int32_t *row_tok,
+                                        const T *__restrict__ E, T *__restrict__ cat, T *__restrict__ cat_lo,
+                                        int H, int V) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  const int i = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
+  if (i >= H) return;
+  const int src = row_src[r];
+  int t = row_tok[r];
+  t = t < 0 ? 0 : (t >= V ? V - 1 : t);
+  const float4 f = *reinterpret_cast<const float4 *>(feat_src + (size_t)src * H + i);
+  const float4 e = load4<T>(E + (size_t)t * H + i);
+  const size_t base = (size_t)r * 2 * H;
+  store_operand4(cat, cat_lo, base + i, f);
+  store_operand4(cat, cat_lo, base + H + i, e);      // the embedding is exact in T: its residual is zero
+}
+
 template <typename T>
 __global__ void cast_rows_kernel(const float *src, const int32_t *row_src,
                                  T *__restrict__ dst, T *__restrict__ dst_lo,
@@ -789,6 +810,12 @@ cudaError_t row_epilogue(Launch L, int dtype, int mode, float *x, SplitIn P, con
 
 cudaError_t eagle_concat(Launch L, int dtype, const float *feat_src, const int32_t *row_src,
                          const int32_t *row_tok, const void *E, Operand cat, int R, int H, int V) {
+  if ((H & 3) == 0) {
+    const int threads = 128;
+    DISPATCH_T(dtype, return launch_k(eagle_concat_vec_kernel<T>, dim3(R, (H / 4 + threads - 1) / threads),
+                                      dim3(threads), 0, L.st, L.pdl, feat_src, row_src, row_tok, (const T *)E,
+                                      (T *)cat.hi, (T *)cat.lo, H, V);)
+  }
   DISPATCH_T(dtype, return launch_k(eagle_concat_kernel<T>, dim3(R), dim3(256), 0, L.st, L.pdl,
                                     feat_src, row_src, row_tok, (const T *)E, (T *)cat.hi, (T *)cat.lo, H,
                                     V);)
