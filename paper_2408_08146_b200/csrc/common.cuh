@@ -137,6 +137,9 @@ cudaError_t eagle_concat(Launch L, int dtype, const float *feat_src, const int32
                          const int32_t *row_tok, const void *E, Operand cat, int R, int H, int V);
 // x <- x + sum(P); xg <- T(x * g) (not normalised); sumsq[r][chunk] <- partial sums of x^2 over
 // chunks of 1024 columns (chunks = ceil(H / 1024)).  H % 4 == 0.
+// x <- E[tok]; xg <- T(x * g) (not normalised); sumsq as in row_update.  H % 4 == 0.
+cudaError_t embed_update(Launch L, int dtype, const int32_t *tok, const void *E, const void *g, float *x,
+                         Operand xg, float *sumsq, int R, int H, int V);
 cudaError_t row_update(Launch L, int dtype, float *x, SplitIn P, const void *g, Operand xg, float *sumsq,
                        int R, int H);
 // q_out: rotated queries in fp32; q_pair (bf16 only, may be null): the same as a bf16 pair

@@ -620,8 +620,15 @@ int koala_verify(koala_ctx *c, const koala_tree *tree) {
   c->pending = RowScale{nullptr, 0, 0.f, 0.f};
   CU_TRY(tree_ancestors(LN(c), c->t, g.B, g.N));
   CU_TRY(plan_verify(LN(c), c->t, c->p, c->seq_len, g.B, g.N, g.head_dim, g.rope_base, g.S_max, c->status));
-  CU_TRY(embed_norm(LN(c), g.dtype, c->p.row_tok, c->embed, c->layers[0].attn_norm, c->x, c->xn, R, g.H, g.V,
-                    g.rms_eps));
+  if ((g.H % 4) == 0 && g.H <= 8192) {
+    // the embedding rows in the deferred form: their RMSNorm scale is applied by the first layer's consumer
+    CU_TRY(embed_update(LN(c), g.dtype, c->p.row_tok, c->embed, c->layers[0].attn_norm, c->x, c->xn, c->sumsq[1],
+                        R, g.H, g.V));
+    c->pending = RowScale{c->sumsq[1], (g.H + 1023) / 1024, 1.f / (float)g.H, g.rms_eps};
+  } else {
+    CU_TRY(embed_norm(LN(c), g.dtype, c->p.row_tok, c->embed, c->layers[0].attn_norm, c->x, c->xn, R, g.H, g.V,
+                      g.rms_eps));
+  }
   const size_t le = kv_layer_elems(g) * c->esz;
   for (int l = 0; l < g.L; ++l) {
     const bool last = l == g.L - 1;

@@ -227,6 +227,31 @@ row_update_kernel(float *__restrict__ x, SplitIn P, const T *__restrict__ g, T *
   if (threadIdx.x == 0) sumsq[(size_t)r * gridDim.x + blockIdx.x] = tot;
 }
 
+// The first rows of a forward in the same deferred form: x <- E[tok]; xg <- T(x * g) (not
+// normalised); sumsq[r][chunk] <- partial sums of x^2.  grid (ceil(H / 1024), R), 256 threads.
+template <typename T>
+__global__ void __launch_bounds__(256)
+embed_update_kernel(const int32_t *tok, const T *__restrict__ E, const T *__restrict__ g, float *__restrict__ x,
+                    T *__restrict__ xg, T *__restrict__ xg_lo, float *__restrict__ sumsq, int H, int V) {
+  __shared__ float red[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.y;
+  const int c = (blockIdx.x * 256 + threadIdx.x) * 4;
+  float ss = 0.f;
+  if (c < H) {
+    int t = tok[r];
+    t = t < 0 ? 0 : (t >= V ? V - 1 : t);
+    const float4 gg = load4<T>(g + c);
+    const float4 o = load4<T>(E + (size_t)t * H + c);
+    *reinterpret_cast<float4 *>(x + (size_t)r * H + c) = o;
+    ss = o.x * o.x + o.y * o.y + o.z * o.z + o.w * o.w;
+    store_operand4(xg, xg_lo, (size_t)r * H + c, make_float4(o.x * gg.x, o.y * gg.y, o.z * gg.z, o.w * gg.w));
+  }
+  const float tot = block_sum(ss, red);
+  if (threadIdx.x == 0) sumsq[(size_t)r * gridDim.x + blockIdx.x] = tot;
+}
+
 // ------------------------------------------------------------------------------- EAGLE fc input
 template <typename T>
 __global__ void eagle_concat_kernel(const float *feat_src,
@@ -830,6 +855,13 @@ cudaError_t cast_rows(Launch L, int dtype, const float *src, const int32_t *row_
 cudaError_t reduce_splits(Launch L, SplitIn P, float *Y, int ldy, int R, int ncols) {
   return launch_k(reduce_splits_kernel, dim3((ncols + 255) / 256, R), dim3(256), 0, L.st, L.pdl, P, Y,
                   ldy, ncols);
+}
+
+cudaError_t embed_update(Launch L, int dtype, const int32_t *tok, const void *E, const void *g, float *x,
+                         Operand xg, float *sumsq, int R, int H, int V) {
+  if (H % 4 != 0) return cudaErrorInvalidValue;
+  DISPATCH_T(dtype, return launch_k(embed_update_kernel<T>, dim3((H + 1023) / 1024, R), dim3(256), 0, L.st, L.pdl,
+                                    tok, (const T *)E, (const T *)g, x, (T *)xg.hi, (T *)xg.lo, sumsq, H, V);)
 }
 
 cudaError_t row_update(Launch L, int dtype, float *x, SplitIn P, const void *g, Operand xg, float *sumsq,
