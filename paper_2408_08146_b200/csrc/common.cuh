@@ -137,6 +137,16 @@ cudaError_t eagle_concat(Launch L, int dtype, const float *feat_src, const int32
                          const int32_t *row_tok, const void *E, Operand cat, int R, int H, int V);
 // x <- x + sum(P); xg <- T(x * g) (not normalised); sumsq[r][chunk] <- partial sums of x^2 over
 // chunks of 1024 columns (chunks = ceil(H / 1024)).  H % 4 == 0.
+// Residual SiLU-Linear blocks of several independent heads in one launch (Medusa-style heads):
+// rows [h * rows_per_head, (h + 1) * rows_per_head) belong to head h, whose partial sums start at
+// P.p = p[h] (row index local to the head) and whose bias is bias[h]:
+// x <- x + SiLU(sum(P) + bias); xn <- T(x).  H % 4 == 0, at most 8 heads.
+struct HeadTab {
+  const void *bias[8];
+  const float *p[8];
+  int rows_per_head;
+};
+cudaError_t resblock_update(Launch L, int dtype, float *x, SplitIn P, HeadTab tab, Operand xn, int R, int H);
 // x <- E[tok]; xg <- T(x * g) (not normalised); sumsq as in row_update.  H % 4 == 0.
 cudaError_t embed_update(Launch L, int dtype, const int32_t *tok, const void *E, const void *g, float *x,
                          Operand xg, float *sumsq, int R, int H, int V);

@@ -62,6 +62,8 @@ struct koala_ctx {
   int attn_chunks;
   float *x, *qbuf, *P, *verify_logits, *draft_logits, *verify_hid, *feat[2], *mx;
   Operand xn, attn_out, act, cat, lmin;
+  size_t p_off;            // floats: where in P the next GEMM's partial sums go (0 except while heads are batched)
+  int p_slots;             // partial matrices that fit there
   Operand qpair;           // rotated queries as a bf16 pair (bf16 configurations)
   float *chain_d;          // [B][D][V] draft distributions of a sampled chain (k = 1 configurations)
   const float *u_draft;    // device [B][D] uniforms: drafted tokens are sampled while non-null
@@ -265,14 +267,15 @@ int do_gemm(koala_ctx *c, Operand X, int K_in, GemmMats m, int R, float *direct,
             SplitIn *out) {
   int ncols = 0;
   for (int i = 0; i < m.n; ++i) ncols += m.n_out[i];
-  float *Y = direct ? direct : c->P;
+  float *Y = direct ? direct : c->P + c->p_off;
   const int ld = direct ? ld_direct : ncols;
   const uint64_t wbytes = (uint64_t)ncols * K_in * c->esz;
   if (c->use_tc && c->cfg.dtype == KOALA_BF16 && tc_supported(m, K_in)) {
     const size_t stride = (size_t)c->Mp * ld;
     const int tb = time_begin(c, KOALA_CLS_GEMM_TC, wbytes);
     SplitIn res;
-    CU_TRY(gemm_tc(LN(c), X, c->Mp, m, K_in, R, Y, ld, direct ? 1 : 0, stride, c->status, MAX_SPLIT, &res));
+    CU_TRY(gemm_tc(LN(c), X, c->Mp, m, K_in, R, Y, ld, direct ? 1 : 0, stride, c->status,
+                   c->p_slots > 0 ? c->p_slots : MAX_SPLIT, &res));
     time_end(c, tb);
     if (out) *out = res;
   } else {
@@ -406,14 +409,43 @@ int draft_medusa(koala_ctx *c) {
   const int R = nh * B;
   CU_TRY(plan_medusa(LN(c), c->t, c->p, B, g.N, nh));
   CU_TRY(cast_rows(LN(c), g.dtype, c->t.pend_hid, c->p.row_src, c->xn, c->mx, 1, R, H));
+  // The heads are independent chains.  Block j of every head is multiplied first (each head's
+  // partial sums in a region of its own), then the heads' epilogues run: the weight stream of one
+  // head's matrix follows the previous head's without a small kernel in between.
+  const size_t region = ((size_t)MAX_SPLIT * c->Mp * c->pcols / (size_t)(nh > 0 ? nh : 1)) & ~(size_t)63;
+  const int slots = (int)(region / ((size_t)c->Mp * H));
+  const bool batched = nh <= 8 && slots >= 1;
+  SplitIn sp[8];
   for (int j = 0; j < g.K; ++j) {
     for (int i = 0; i < nh; ++i) {
-      SplitIn s;
       GemmMats m{{c->res_w[(size_t)i * g.K + j], nullptr, nullptr}, {H, 0, 0}, 1};
       const size_t off = (size_t)i * B * H * c->esz;
       Operand xi{(unsigned char *)c->xn.hi + off, c->xn.lo ? (unsigned char *)c->xn.lo + off : nullptr};
-      K_TRY(do_gemm(c, xi, H, m, B, nullptr, 0, &s));
+      if (batched) { c->p_off = (size_t)i * region; c->p_slots = slots < MAX_SPLIT ? slots : MAX_SPLIT; }
+      SplitIn s;
+      const int rc = do_gemm(c, xi, H, m, B, nullptr, 0, &s);
+      c->p_off = 0;
+      c->p_slots = 0;
+      if (rc != KOALA_OK) return rc;
+      if (batched) { sp[i] = s; continue; }
       CU_TRY(row_epilogue(LN(c), g.dtype, 2, c->mx + (size_t)i * B * H, s, c->res_b[(size_t)i * g.K + j],
+                          nullptr, xi, nullptr, B, H, g.rms_eps));
+    }
+    if (!batched) continue;
+    bool same = (H % 4) == 0 && (sp[0].ld % 4) == 0 && (sp[0].stride % 4) == 0 && sp[0].sk_ctas == 0;
+    for (int i = 1; i < nh; ++i) same = same && sp[i].n == sp[0].n && sp[i].stride == sp[0].stride && sp[i].ld == sp[0].ld;
+    if (same) {            // one launch finishes block j of every head
+      HeadTab tab;
+      memset(&tab, 0, sizeof(tab));
+      for (int i = 0; i < nh; ++i) { tab.bias[i] = c->res_b[(size_t)i * g.K + j]; tab.p[i] = sp[i].p; }
+      tab.rows_per_head = B;
+      CU_TRY(resblock_update(LN(c), g.dtype, c->mx, sp[0], tab, c->xn, R, H));
+      continue;
+    }
+    for (int i = 0; i < nh; ++i) {
+      const size_t off = (size_t)i * B * H * c->esz;
+      Operand xi{(unsigned char *)c->xn.hi + off, c->xn.lo ? (unsigned char *)c->xn.lo + off : nullptr};
+      CU_TRY(row_epilogue(LN(c), g.dtype, 2, c->mx + (size_t)i * B * H, sp[i], c->res_b[(size_t)i * g.K + j],
                           nullptr, xi, nullptr, B, H, g.rms_eps));
     }
   }
@@ -459,6 +491,8 @@ int koala_init(const koala_config *cfg, const koala_weights *w, const koala_stat
   c->poll_pending = false;
   c->last_status = 0;
   c->u_draft = nullptr;
+  c->p_off = 0;
+  c->p_slots = 0;
   char why[128];
   if (!config_ok(cfg, why, sizeof(why))) return fail(c, KOALA_E_INVALID, "%s", why);
   if (!w || !st) return fail(c, KOALA_E_INVALID, "null weights or state");

@@ -227,6 +227,26 @@ row_update_kernel(float *__restrict__ x, SplitIn P, const T *__restrict__ g, T *
   if (threadIdx.x == 0) sumsq[(size_t)r * gridDim.x + blockIdx.x] = tot;
 }
 
+template <typename T>
+__global__ void __launch_bounds__(256)
+resblock_update_kernel(float *__restrict__ x, SplitIn P, HeadTab tab, T *__restrict__ xn, T *__restrict__ xn_lo, int H) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.y;
+  const int c = (blockIdx.x * 256 + threadIdx.x) * 4;
+  if (c >= H) return;
+  const int head = r / tab.rows_per_head;
+  P.p = tab.p[head];
+  const float4 p = split_sum4(P, r - head * tab.rows_per_head, c);
+  const float4 b = load4<T>(reinterpret_cast<const T *>(tab.bias[head]) + c);
+  float *xr = x + (size_t)r * H + c;
+  const float4 xv = *reinterpret_cast<const float4 *>(xr);
+  const float4 o = make_float4(xv.x + silu_f(p.x + b.x), xv.y + silu_f(p.y + b.y), xv.z + silu_f(p.z + b.z),
+                               xv.w + silu_f(p.w + b.w));
+  *reinterpret_cast<float4 *>(xr) = o;
+  store_operand4(xn, xn_lo, (size_t)r * H + c, o);
+}
+
 // The first rows of a forward in the same deferred form: x <- E[tok]; xg <- T(x * g) (not
 // normalised); sumsq[r][chunk] <- partial sums of x^2.  grid (ceil(H / 1024), R), 256 threads.
 template <typename T>
@@ -855,6 +875,12 @@ cudaError_t cast_rows(Launch L, int dtype, const float *src, const int32_t *row_
 cudaError_t reduce_splits(Launch L, SplitIn P, float *Y, int ldy, int R, int ncols) {
   return launch_k(reduce_splits_kernel, dim3((ncols + 255) / 256, R), dim3(256), 0, L.st, L.pdl, P, Y,
                   ldy, ncols);
+}
+
+cudaError_t resblock_update(Launch L, int dtype, float *x, SplitIn P, HeadTab tab, Operand xn, int R, int H) {
+  if (H % 4 != 0 || P.ld % 4 != 0 || P.stride % 4 != 0 || tab.rows_per_head < 1) return cudaErrorInvalidValue;
+  DISPATCH_T(dtype, return launch_k(resblock_update_kernel<T>, dim3((H + 1023) / 1024, R), dim3(256), 0, L.st, L.pdl,
+                                    x, P, tab, (T *)xn.hi, (T *)xn.lo, H);)
 }
 
 cudaError_t embed_update(Launch L, int dtype, const int32_t *tok, const void *E, const void *g, float *x,
