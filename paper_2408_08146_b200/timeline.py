@@ -50,7 +50,7 @@ def main():
             eng.step(forced)
         torch.cuda.synchronize()
     ks = sorted([(e.time_range.start, e.time_range.end, e.name) for e in prof.events() if "koala" in e.name])
-    first = [i for i, k in enumerate(ks) if "embed_norm" in k[2]]          # one per verify call
+    first = [i for i, k in enumerate(ks) if "embed_update" in k[2] or "embed_norm" in k[2]]   # one per verify call
     seg = ks[first[1]:first[2]]
     print(f"step span {ks[first[2]][0] - ks[first[1]][0]:.1f} us, {len(seg)} kernels")
     latest, inc = None, {}
