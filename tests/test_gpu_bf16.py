@@ -188,3 +188,9 @@ def test_t13_eagle_batch4_ragged():
 def test_t33_eagle_shape(K):
     """33B-shaped layers (hidden 6656, 52 heads, FFN 17920) with a deeper head; one target layer."""
     _teacher_forced_iteration(reduced(T33_EAGLE, 1, K=K, S_max=640, prompt_len=512))
+
+
+def test_ragged_vocabulary_and_odd_top_k():
+    """A vocabulary that is no multiple of the top-k kernel's parts or of the GEMM's 128-row tiles, k = 7."""
+    _teacher_forced_iteration(reduced(T7_EAGLE, 1, K=1, V=5003 - 3, topk=7, N=40, S_max=384, prompt_len=256))
+    _teacher_forced_iteration(reduced(T7_EAGLE, 1, K=1, V=32768, topk=16, D=2, N=64, S_max=384, prompt_len=256))
