@@ -710,6 +710,7 @@ topk_logp_fast_kernel(const float *logits, int32_t *__restrict__ tok, float *__r
 constexpr int TKP = 8;            // CTAs per row
 __global__ void __launch_bounds__(256)
 topk_logp_cluster_kernel(const float *logits, int32_t *__restrict__ tok, float *__restrict__ logp, int V, int k) {
+  // logp == nullptr: only the ids are wanted (the arg-max of a row is its top-1), no exponentials
   __shared__ ValIdx cand[8 * 32];
   __shared__ ValIdx mine[32];     // this CTA's k best, read by CTA 0
   __shared__ float s_ms[2];       // this CTA's (max, sum of exp(v - max))
@@ -735,7 +736,7 @@ topk_logp_cluster_kernel(const float *logits, int32_t *__restrict__ tok, float *
   mx = warp_max(lane < 8 ? redf[lane] : -INFINITY);
   __syncthreads();
   float se = 0.f;
-  if (mx != -INFINITY) {
+  if (mx != -INFINITY && logp != nullptr) {
 #pragma unroll
     for (int j = 0; j < 16; ++j) se += expf(vals[j] - mx);
   }
@@ -807,7 +808,7 @@ topk_logp_cluster_kernel(const float *logits, int32_t *__restrict__ tok, float *
         if (c8[j].i == win.i) c8[j] = ValIdx{-INFINITY, 0x7fffffff};
       if (lane == 0) {
         tok[(size_t)r * k + rnd] = win.i;
-        logp[(size_t)r * k + rnd] = win.v - lse;
+        if (logp != nullptr) logp[(size_t)r * k + rnd] = win.v - lse;
       }
     }
   }
@@ -941,28 +942,32 @@ cudaError_t tree_attention(Launch L, int dtype, const float *q, const void *k_ca
   return cudaErrorInvalidValue;
 }
 
+static cudaError_t topk_cluster_launch(Launch L, const float *logits, int32_t *tok, float *logp, int R, int V, int k) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(TKP, R);
+  cfg.blockDim = dim3(256);
+  cfg.stream = L.st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = L.pdl ? 1 : 0;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = TKP;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  ++g_launches;
+  return cudaLaunchKernelEx(&cfg, topk_logp_cluster_kernel, logits, tok, logp, V, k);
+}
+
 cudaError_t argmax_rows(Launch L, const float *logits, int32_t *out, int R, int V) {
+  // the arg-max (ties: smaller id) is the top-1; wide rows go to the eight-CTA kernel
+  if (V <= 32768 && V >= 4096) return topk_cluster_launch(L, logits, out, nullptr, R, V, 1);
   return launch_k(argmax_rows_kernel, dim3(R), dim3(1024), 0, L.st, L.pdl, logits, out, V);
 }
 
 cudaError_t topk_logp(Launch L, const float *logits, int32_t *tok, float *logp, int R, int V, int k) {
-  if (V <= 32768 && k <= 32 && V >= 4096) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(TKP, R);
-    cfg.blockDim = dim3(256);
-    cfg.stream = L.st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = L.pdl ? 1 : 0;
-    attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = TKP;
-    attr[1].val.clusterDim.y = 1;
-    attr[1].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    ++g_launches;
-    return cudaLaunchKernelEx(&cfg, topk_logp_cluster_kernel, logits, tok, logp, V, k);
-  }
+  if (V <= 32768 && k <= 32 && V >= 4096) return topk_cluster_launch(L, logits, tok, logp, R, V, k);
   if (V <= 32768 && k <= 32)
     return launch_k(topk_logp_fast_kernel, dim3(R), dim3(1024), 0, L.st, L.pdl, logits, tok, logp, V, k);
   const size_t smem = (size_t)V * sizeof(float);
