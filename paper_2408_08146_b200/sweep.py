@@ -24,7 +24,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from workloads import T33_EAGLE, T7_EAGLE, T7_MEDUSA  # noqa: E402
+from workloads import T13_EAGLE, T33_EAGLE, T7_EAGLE, T7_MEDUSA  # noqa: E402
 from workloads.generate import WeightStore, medusa_static_tree, uniform_ints  # noqa: E402
 
 from . import Koala  # noqa: E402
@@ -197,14 +197,25 @@ def main():
     ap.add_argument("--what", default="draft,verify")
     ap.add_argument("--reps", type=int, default=10)
     ap.add_argument("--json", default="")
-    ap.add_argument("--model", default="7b", choices=["7b", "33b"],
-                    help="33b: the 33B shape (65 GB of weights): draft K = 1..8, verify at three points")
+    ap.add_argument("--model", default="7b", choices=["7b", "13b", "33b"],
+                    help="13b: the 13B shape at batch 1 and 4 (tree 64, context 2048); "
+                         "33b: the 33B shape (65 GB of weights): draft K = 1..8, verify at three points")
     args = ap.parse_args()
     peak, tflops, src = measured_peak()
     print(f"HBM peak {peak:.0f} GB/s ({src}); nominal {NOMINAL_GBS:.0f} GB/s")
     out = {"peak_GBps": peak, "peak_source": src}
     if "medusa" in args.what:
         out["medusa"] = medusa_sweep(args.reps, peak)
+    if args.model == "13b":
+        store = WeightStore(T13_EAGLE.with_(K=2), DEV)
+        if "draft" in args.what:
+            out["draft"] = draft_sweep(store, args.reps, peak, T13_EAGLE, (1, 2))
+        if "verify" in args.what:
+            out["verify"] = verify_sweep(store, args.reps, peak, tflops, T13_EAGLE,
+                                         [(64, 512, 1), (64, 2048, 1), (64, 2048, 4)])
+        if args.json:
+            json.dump(out, open(args.json, "w"), indent=1)
+        return
     if args.model == "33b":
         store = WeightStore(T33_EAGLE.with_(K=8), DEV)
         if "draft" in args.what:
