@@ -1,7 +1,7 @@
 """Times the library's weight-streaming GEMM on the decoder shapes (kernel sweep).
 
     python -m paper_2408_08146_b200.gemm_bench [--model 7b|13b] [--tokens 64] [--shapes qkv,o,...]
-                                               [--splits 0,1,3] [--stages 0] [--plain] [--iters 20]
+                                               [--splits 0,1,3] [--stages 0] [--plain] [--iters 20] [--tune key=value,...]
 
 Prints, per shape and split-K factor, the mean time of one call (CUDA events around `iters`
 back-to-back calls that rotate over enough weight copies to defeat the L2) and the weight bytes
@@ -34,6 +34,7 @@ def main():
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--plain", action="store_true", help="plain bf16 activations instead of value+residual pairs")
     ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--tune", default="", help="tuning keys of koala_set_tuning, e.g. 2=4,3=1")
     args = ap.parse_args()
     lib = binding.load_library()
     dev = "cuda:0"
@@ -41,6 +42,9 @@ def main():
     pair = 0 if args.plain else 1
     rows = lib.koala_gemm_x_rows(M, pair)
     lib.koala_set_tuning(1, args.stages)
+    for kv in filter(None, args.tune.split(",")):
+        k, v = kv.split("=")
+        lib.koala_set_tuning(int(k), int(v))
     st = torch.cuda.current_stream().cuda_stream
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     for name in args.shapes.split(","):
