@@ -317,6 +317,7 @@ int g_tune_no_streamk = 0;  // 1 = always the per-tile decomposition
 int g_tune_l2_ahead = -1;   // < 0 = default
 int g_tune_late_w = 0;      // 1 = weights wait for the dependency too
 int g_tune_early_stages = -1; // < 0 = all stages
+int g_tune_no_wave_split = 0; // 1 = several token tiles keep the one-wave rule's split factor
 int g_tune_traffic_div = 8; // split <= K_in / (div * tokens)
 
 bool get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out) {
@@ -376,6 +377,7 @@ void attn_tc_set_min_rows(int rows);
 void tc_set_tuning(int key, int value) {
   if (key == 9) attn_tc_set_min_rows(value);
   if (key == 1) g_tune_stages = value;
+  if (key == 10) g_tune_no_wave_split = value;
   if (key == 2) g_tune_max_split = value;
   if (key == 3) g_tune_no_streamk = value;
   if (key == 5) g_tune_l2_ahead = value;
@@ -399,16 +401,40 @@ bool tc_supported(const GemmMats &m, int K_in) {
 // Split-K factor: as many CTAs as fit in one wave of the co-resident slots (two per SM), while
 // every split keeps at least 8 K-blocks and the fp32 partial sums written and re-read
 // (split x tokens x 4 bytes per output) stay below about half of the weight bytes.
-int tc_default_split(int n_tiles, int kblocks, int tokens) {
-  const int slots = 2 * g_num_sms;
-  int s = slots / (n_tiles > 0 ? n_tiles : 1);
+static int split_cap(int kblocks, int tokens) {
+  int s = 8;
   const int by_k = kblocks / 8;
   const int by_traffic = (kblocks * 64) / (g_tune_traffic_div * (tokens > 0 ? tokens : 1));
   if (s > by_k) s = by_k;
   if (s > by_traffic) s = by_traffic;
-  if (s > 8) s = 8;
   if (g_tune_max_split > 0 && s > g_tune_max_split) s = g_tune_max_split;
   return s < 1 ? 1 : s;
+}
+
+int tc_default_split(int n_tiles, int kblocks, int tokens) {
+  const int slots = 2 * g_num_sms;
+  int s = slots / (n_tiles > 0 ? n_tiles : 1);
+  const int cap = split_cap(kblocks, tokens);
+  if (s > cap) s = cap;
+  return s < 1 ? 1 : s;
+}
+
+// Several token tiles (more than 128 rows as pairs): `ctas` = weight tiles x token tiles may exceed
+// the co-resident slots, and then the launch runs in rounds whose last one can be nearly empty.
+// The time goes as rounds(split) / split (each CTA covers K / split), so among the allowed factors
+// take the one with the fewest round-lengths, but leave `split0` (the one-wave rule's choice)
+// unless another is at least 10 % better.
+static int wave_split(int ctas, int kblocks, int tokens, int split0) {
+  const int slots = 2 * g_num_sms;
+  const int cap = split_cap(kblocks, tokens);
+  auto cost = [&](int sp) { return (double)((ctas * sp + slots - 1) / slots) / sp; };
+  int best = split0 <= cap ? split0 : cap;
+  if (best < 1) best = 1;
+  double best_cost = cost(best);
+  const double keep = 0.9 * best_cost;
+  for (int sp = 1; sp <= cap; ++sp)
+    if (cost(sp) < keep && cost(sp) < best_cost - 1e-9) { best = sp; best_cost = cost(sp); }
+  return best;
 }
 
 // Stream-K plan: how many CTAs share the (tile, K-block) units.  At most two per SM, at least 8
@@ -490,7 +516,10 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   }
   if (!sk) {
     sk_ctas = 0;
-    if (split < 1) split = tc_default_split(n_tiles, P.kblocks, R);
+    if (split < 1) {
+      split = tc_default_split(n_tiles, P.kblocks, R);
+      if (ztiles > 1 && !g_tune_no_wave_split) split = wave_split(n_tiles * ztiles, P.kblocks, R, split);
+    }
     if (split > P.kblocks) split = P.kblocks;
     if (max_slots > 0 && split > max_slots) split = max_slots;
   }
