@@ -253,7 +253,8 @@ int koala_timing_read(koala_ctx *ctx, koala_timing *out);
  * pipeline (< 0 = default 0); key 6 = 1 delays the weight stream until the previous kernel has
  * finished; key 7 = divisor of the split-K partial-sum traffic bound (default 8); key 8 = how many
  * pipeline stages request their weight tile before that wait (< 0 = all, the default); key 10 = 1
- * keeps the one-wave split-K factor when a launch has several token tiles (more than 128 rows). */
+ * keeps the one-wave split-K factor when a launch has several token tiles (more than 128 rows);
+ * key 11 = 1 keeps 128 weight rows per CTA also for the widest token tiles (MMA N = 256). */
 void koala_set_tuning(int key, int value);
 
 /* Kernels launched by the library in this process so far (all contexts). */

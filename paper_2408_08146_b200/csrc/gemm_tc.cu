@@ -14,6 +14,11 @@
 // token tile then holds the hi rows followed by the lo rows of the same tokens (MMA N doubles),
 // and the epilogue adds the two halves of the accumulator, so the product carries 16 significant
 // bits of the activations at no extra weight traffic.
+// Wide token tiles (MMA N = 256: more than 64 tokens as pairs): a pipeline stage would be 16 KB of
+// weights + 32 KB of activations, and the ring is bound by its capacity (bytes in flight /
+// latency), two thirds of it activations.  There a CTA takes 256 weight rows instead: two MMAs per
+// K step share the activation tile and fill two accumulators (all 512 tensor-memory columns), a
+// stage is 32 + 32 KB, one CTA per SM with three stages keeps 1.5 times the weight bytes in flight.
 // Split-K: grid.y CTAs share a weight tile and write separate partial outputs that the consumer
 // kernel sums in a fixed order (deterministic).
 // Every wait is bounded: on expiry the kernel records KOALA_E_TIMEOUT in *status, drains, frees
@@ -60,6 +65,7 @@ struct TcParams {
   unsigned sk_units;  // tiles * kblocks
   size_t split_stride;
   int stages;
+  int wide;           // 1: 256 weight rows per CTA (two accumulators), N = 256, one CTA per SM
   int early_w;        // how many of the first stages' weight tiles are requested before the dependency wait
   int l2_ahead;       // weight tiles prefetched into L2 beyond the ring before the dependency wait
   int *status;
@@ -86,7 +92,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char *tiles = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
   const int x_stage_bytes = P.bn * BK * 2;
-  const int stage_bytes = W_STAGE_BYTES + x_stage_bytes;   // both multiples of 1024
+  const int w_stage_bytes = P.wide ? 2 * W_STAGE_BYTES : W_STAGE_BYTES;
+  const int stage_bytes = w_stage_bytes + x_stage_bytes;   // both multiples of 1024
+  const int bm = P.wide ? 2 * BM : BM;                     // weight rows per tile
   const int KB = P.kblocks;
 
   // this CTA's run of (tile, K-block) units, tile-major; a run may cross tile boundaries (stream-K)
@@ -105,10 +113,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 
   // weight tensor map and first row of a tile
   auto tile_map = [&](int tile, int &row0) -> const CUtensorMap * {
-    if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * BM; return &tmW2; }
-    if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * BM; return &tmW1; }
-    row0 = tile * BM;
+    if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * bm; return &tmW2; }
+    if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * bm; return &tmW1; }
+    row0 = tile * bm;
     return &tmW0;
+  };
+  // one weight tile of a stage: 128 rows per copy
+  auto load_w = [&](const CUtensorMap *tmW, uint64_t *bar, unsigned char *dst, int kb, int row0) {
+    tma_load_2d(tmW, bar, dst, kb * BK, row0);
+    if (P.wide) tma_load_2d(tmW, bar, dst + W_STAGE_BYTES, kb * BK, row0 + BM);
   };
   const int pre = n_units < P.stages ? n_units : P.stages;
 
@@ -136,10 +149,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     for (int it = 0; it < ahead; ++it) {
       if (it < early) {
         mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
-        tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, kb * BK, row0);
+        load_w(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, kb, row0);
       } else {
         asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
                      ::"l"(tmW), "r"(kb * BK), "r"(row0) : "memory");
+        if (P.wide)
+          asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+                       ::"l"(tmW), "r"(kb * BK), "r"(row0 + BM) : "memory");
       }
       if (++kb == KB) { kb = 0; ++tile; tmW = tile_map(tile, row0); }
     }
@@ -148,7 +164,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)(P.tmem_cols * P.nbuf))
+                 ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)(P.tmem_cols * P.nbuf * (P.wide ? 2 : 1)))
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -168,10 +184,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       kb = (int)(u_lo % KB);
       tmW = tile_map(tile, row0);
       for (int it = 0; it < pre; ++it) {
-        unsigned char *xd = tiles + (size_t)it * stage_bytes + W_STAGE_BYTES;
+        unsigned char *xd = tiles + (size_t)it * stage_bytes + w_stage_bytes;
         if (it >= P.early_w) {
           mbar_expect_tx(&full_bar[it], (uint32_t)stage_bytes);
-          tma_load_2d(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, kb * BK, row0);
+          load_w(tmW, &full_bar[it], tiles + (size_t)it * stage_bytes, kb, row0);
         }
         tma_load_2d(&tmX, &full_bar[it], xd, kb * BK, tok0);
         if (P.pair) tma_load_2d(&tmXlo, &full_bar[it], xd + lo_off, kb * BK, tok0);
@@ -185,9 +201,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         if (!ok) break;
         mbar_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
         unsigned char *dst = tiles + (size_t)s * stage_bytes;
-        tma_load_2d(tmW, &full_bar[s], dst, kb * BK, row0);
-        tma_load_2d(&tmX, &full_bar[s], dst + W_STAGE_BYTES, kb * BK, tok0);
-        if (P.pair) tma_load_2d(&tmXlo, &full_bar[s], dst + W_STAGE_BYTES + lo_off, kb * BK, tok0);
+        load_w(tmW, &full_bar[s], dst, kb, row0);
+        tma_load_2d(&tmX, &full_bar[s], dst + w_stage_bytes, kb * BK, tok0);
+        if (P.pair) tma_load_2d(&tmXlo, &full_bar[s], dst + w_stage_bytes + lo_off, kb * BK, tok0);
         if (++kb == KB) { kb = 0; ++tile; tmW = tile_map(tile, row0); }
         if (++s == P.stages) { s = 0; ph ^= 1u; }
       }
@@ -220,13 +236,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t wa = smem_u32(tiles + (size_t)s * stage_bytes);
         const uint64_t da = smem_desc_sw128(wa);
-        const uint64_t db = smem_desc_sw128(wa + W_STAGE_BYTES);
+        const uint64_t da2 = smem_desc_sw128(wa + W_STAGE_BYTES);      // wide: the second 128 weight rows
+        const uint64_t db = smem_desc_sw128(wa + (uint32_t)w_stage_bytes);
         const uint32_t dacc = tmem_acc + (uint32_t)(buf * P.tmem_cols);
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; ++k) {
           // advance 32 bytes (16 bf16) inside the swizzled row: +2 in the 16-byte address field
           umma_bf16(dacc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
                     (!seg_start || k > 0) ? 1u : 0u);
+          if (P.wide)
+            umma_bf16(dacc + (uint32_t)P.tmem_cols, da2 + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
+                      (!seg_start || k > 0) ? 1u : 0u);
         }
         umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
         const bool seg_end = (kb == KB - 1) || it == n_units - 1;
@@ -257,16 +277,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       int row0, col_off = 0, n_rows = P.n0;
-      if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * BM; col_off = P.n0 + P.n1; n_rows = P.n2; }
-      else if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * BM; col_off = P.n0; n_rows = P.n1; }
-      else row0 = tile * BM;
+      if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * bm; col_off = P.n0 + P.n1; n_rows = P.n2; }
+      else if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * bm; col_off = P.n0; n_rows = P.n1; }
+      else row0 = tile * bm;
       // which partial-sum slot: classic = the split index; stream-K = rank among the tile's contributors
       int slot = blockIdx.y;
       if (P.sk_ctas > 0)
         slot = (int)blockIdx.x - (int)sk_owner((unsigned)tile * KB, (unsigned)P.sk_ctas, P.sk_units);
-      const int feat = row0 + quarter * 32 + lane;
+      for (int hw = 0; hw < (P.wide ? 2 : 1); ++hw) {      // wide: one accumulator per 128 weight rows
+      const int feat = row0 + hw * BM + quarter * 32 + lane;
       float *Yp = P.Y + (size_t)slot * P.split_stride + col_off + feat;
-      const uint32_t lane_base = tmem_acc + (uint32_t)(buf * P.tmem_cols) + ((uint32_t)(quarter * 32) << 16);
+      const uint32_t lane_base = tmem_acc + (uint32_t)((buf + hw) * P.tmem_cols) + ((uint32_t)(quarter * 32) << 16);
       for (int c0 = 0; c0 < P.tt; c0 += 16) {
         uint32_t v[16], w[16];
         tmem_ld16(lane_base + (uint32_t)c0, v);
@@ -282,6 +303,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
           }
         }
       }
+      }
       // hand the accumulator buffer back to the MMA issuer
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -295,7 +317,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
-                 ::"r"(tmem_acc), "r"((uint32_t)(P.tmem_cols * P.nbuf))
+                 ::"r"(tmem_acc), "r"((uint32_t)(P.tmem_cols * P.nbuf * (P.wide ? 2 : 1)))
                  : "memory");
   }
   if (threadIdx.x == 0 && s_error && P.status) atomicMax(P.status, E_TIMEOUT);
@@ -318,6 +340,7 @@ int g_tune_l2_ahead = -1;   // < 0 = default
 int g_tune_late_w = 0;      // 1 = weights wait for the dependency too
 int g_tune_early_stages = -1; // < 0 = all stages
 int g_tune_no_wave_split = 0; // 1 = several token tiles keep the one-wave rule's split factor
+int g_tune_no_wide = 0;      // 1 = 128 weight rows per CTA also for wide token tiles
 int g_tune_traffic_div = 8; // split <= K_in / (div * tokens)
 
 bool get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out) {
@@ -378,6 +401,7 @@ void tc_set_tuning(int key, int value) {
   if (key == 9) attn_tc_set_min_rows(value);
   if (key == 1) g_tune_stages = value;
   if (key == 10) g_tune_no_wave_split = value;
+  if (key == 11) g_tune_no_wide = value;
   if (key == 2) g_tune_max_split = value;
   if (key == 3) g_tune_no_streamk = value;
   if (key == 5) g_tune_l2_ahead = value;
@@ -424,8 +448,7 @@ int tc_default_split(int n_tiles, int kblocks, int tokens) {
 // The time goes as rounds(split) / split (each CTA covers K / split), so among the allowed factors
 // take the one with the fewest round-lengths, but leave `split0` (the one-wave rule's choice)
 // unless another is at least 10 % better.
-static int wave_split(int ctas, int kblocks, int tokens, int split0) {
-  const int slots = 2 * g_num_sms;
+static int wave_split(int ctas, int kblocks, int tokens, int split0, int slots) {
   const int cap = split_cap(kblocks, tokens);
   auto cost = [&](int sp) { return (double)((ctas * sp + slots - 1) / slots) / sp; };
   int best = split0 <= cap ? split0 : cap;
@@ -488,9 +511,14 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   P.R = R;
   P.bn = bn;
   P.tmem_cols = cols;
-  const int t0 = (m.n_out[0] + BM - 1) / BM;
-  const int t1 = m.n > 1 ? (m.n_out[1] + BM - 1) / BM : 0;
-  const int t2 = m.n > 2 ? (m.n_out[2] + BM - 1) / BM : 0;
+  // wide mode: N = 256, every matrix a whole number of 256-row tiles, room for three 64 KB stages
+  bool wide = !g_tune_no_wide && bn == 256 && g_smem_optin - 2048 >= 3 * (2 * W_STAGE_BYTES + bn * BK * 2);
+  for (int i = 0; i < m.n && wide; ++i) wide = (m.n_out[i] % (2 * BM)) == 0;
+  const int bmw = wide ? 2 * BM : BM;
+  P.wide = wide ? 1 : 0;
+  const int t0 = (m.n_out[0] + bmw - 1) / bmw;
+  const int t1 = m.n > 1 ? (m.n_out[1] + bmw - 1) / bmw : 0;
+  const int t2 = m.n > 2 ? (m.n_out[2] + bmw - 1) / bmw : 0;
   const int n_tiles = t0 + t1 + t2;
   P.tiles0 = t0;
   P.tiles1 = t0 + t1;
@@ -500,7 +528,7 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   P.kblocks = K_in / BK;
   // stream-K (split == 0): needs a single token tile and 128-row-aligned matrices, so that a
   // column's tile (and with it the number of partial sums to add) follows from the column index
-  bool sk = split == 0 && ztiles == 1 && max_slots >= 2 && out != nullptr && !g_tune_no_streamk;
+  bool sk = split == 0 && ztiles == 1 && max_slots >= 2 && out != nullptr && !g_tune_no_streamk && !wide;
   for (int i = 0; i < m.n && sk; ++i) sk = (m.n_out[i] % BM) == 0;
   // stream-K pays off where the per-tile decomposition cannot be split further and leaves the SMs
   // unevenly loaded (more tiles than SMs, not a whole number of two-per-SM waves); elsewhere
@@ -516,9 +544,12 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   }
   if (!sk) {
     sk_ctas = 0;
-    if (split < 1) {
+    if (split < 1 && wide) {
+      // one CTA per SM: the factor with the fewest round-lengths over the SMs
+      split = wave_split(n_tiles * ztiles, P.kblocks, R, 1, g_num_sms);
+    } else if (split < 1) {
       split = tc_default_split(n_tiles, P.kblocks, R);
-      if (ztiles > 1 && !g_tune_no_wave_split) split = wave_split(n_tiles * ztiles, P.kblocks, R, split);
+      if (ztiles > 1 && !g_tune_no_wave_split) split = wave_split(n_tiles * ztiles, P.kblocks, R, split, 2 * g_num_sms);
     }
     if (split > P.kblocks) split = P.kblocks;
     if (max_slots > 0 && split > max_slots) split = max_slots;
@@ -529,14 +560,14 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   P.split_stride = split_stride;
   P.status = status;
   P.nbuf = (sk && 2 * cols <= 256) ? 2 : 1;
-  const int stage_bytes = W_STAGE_BYTES + bn * BK * 2;
+  const int stage_bytes = (wide ? 2 : 1) * W_STAGE_BYTES + bn * BK * 2;
   int stages = (g_smem_optin - 2048) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages > 8) stages = 8;
   // default: two CTAs per SM (each with half of the shared memory), so that one CTA's prologue and
   // epilogue overlap the other's streaming
   const int two_per_sm = (g_smem_optin / 2 - 2048) / stage_bytes;
-  if (g_tune_stages == 0 && two_per_sm >= 2 && two_per_sm < stages) stages = two_per_sm;
+  if (g_tune_stages == 0 && two_per_sm >= 2 && two_per_sm < stages && !wide) stages = two_per_sm;
   if (g_tune_stages > 0 && g_tune_stages < stages) stages = g_tune_stages;
   if (stages < 2) return cudaErrorInvalidValue;
   P.stages = stages;
