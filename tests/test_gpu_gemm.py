@@ -10,7 +10,8 @@ pytestmark = pytest.mark.gpu
 
 SHAPES = [  # (tokens, out features, in features)
     (1, 128, 64), (10, 4096, 4096), (16, 256, 128), (17, 200, 192), (60, 1536, 4096),
-    (64, 384, 11008), (40, 640, 5120), (256, 256, 1024), (300, 256, 512), (6, 32000, 4096)]
+    (64, 384, 11008), (40, 640, 5120), (256, 256, 1024), (300, 256, 512), (6, 32000, 4096),
+    (250, 1280, 2048)]      # 256-row weight tiles (N = 256), several of them, ragged token tile
 
 
 def _inputs(M, N, K):
@@ -46,7 +47,7 @@ def test_cuda_core_gemm(shape):
 
 
 @pytest.mark.parametrize("shape", [(10, 4096, 4096), (60, 1536, 4096), (100, 256, 11008), (130, 384, 512),
-                                   (256, 256, 1024)])
+                                   (256, 256, 1024), (128, 512, 4096), (200, 1024, 2048), (120, 768, 1024)])
 @pytest.mark.parametrize("tc", [True, False], ids=["tensor_core", "cuda_core"])
 def test_gemm_with_activation_pairs(shape, tc):
     """fp32 activations given as a bf16 value + bf16 rounding residual: the product must be that of
