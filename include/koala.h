@@ -23,8 +23,8 @@
  *   - Matrices are row-major [out][in].  "dtype" is the storage type of weights, KV caches and
  *     matrix-multiply operands (fp32 or bf16); accumulation, softmax, norms and the residual
  *     stream are fp32 in both cases.  With bf16 the activations entering a matrix multiply are
- *     kept as two bf16 values (the rounded value and its rounding residual) unless
- *     KOALA_F_BF16_ACTIVATIONS is set, so only the weights and the KV cache are rounded to bf16.
+ *     kept as two bf16 values (the rounded value and its rounding residual), so only the weights
+ *     and the KV cache are rounded to bf16.
  *   - KV caches are laid out [layer][B][n_heads][S_max][head_dim].
  *   - A tree has at most N nodes per sequence, node 0 the root, parent index < child index.
  *     Node u of sequence b is row b*N + u of every per-node buffer.
@@ -56,10 +56,6 @@ extern "C" {
 /* flags */
 #define KOALA_F_NO_TENSOR_CORES 1u /* run every GEMM on the CUDA-core path (debugging / A-B checks) */
 #define KOALA_F_NO_PDL 2u          /* launch kernels without programmatic dependent launch         */
-#define KOALA_F_BF16_ACTIVATIONS 4u /* bf16 only: round matrix-multiply inputs to plain bf16 instead of
-                                       keeping them as a bf16 pair (value + rounding residual); halves
-                                       the tensor-core work, costs about 1e-2 relative accuracy over a
-                                       32-layer forward */
 
 #define KOALA_MAX_TREE 128 /* largest N: ancestor sets are 128-bit masks */
 #define KOALA_MAX_TOPK 16
@@ -246,20 +242,6 @@ typedef struct {
 } koala_timing;
 int koala_timing_read(koala_ctx *ctx, koala_timing *out);
 
-/* Process-wide tuning of the tensor-core matrix multiply (for sweeps; the defaults are chosen
- * for B200): key 1 = shared-memory pipeline stages per CTA (0 = as many as fit, at most 8);
- * key 2 = upper bound on the automatic split-K factor (0 = default); key 3 = 1 switches stream-K
- * off (every CTA stays inside one weight tile); key 5 = weight tiles prefetched into L2 ahead of the
- * pipeline (< 0 = default 0); key 6 = 1 delays the weight stream until the previous kernel has
- * finished; key 7 = divisor of the split-K partial-sum traffic bound (default 8); key 8 = how many
- * pipeline stages request their weight tile before that wait (< 0 = all, the default); key 10 = 1
- * keeps the one-wave split-K factor when a launch has several token tiles (more than 128 rows);
- * key 11 = 1 keeps 128 weight rows per CTA also for the widest token tiles (MMA N = 256). */
-void koala_set_tuning(int key, int value);
-
-/* Kernels launched by the library in this process so far (all contexts). */
-uint64_t koala_launch_count(void);
-
 /* Non-blocking: *done = 1 if everything enqueued so far has finished; *device_status = the
  * device status word as of the last finished poll copy (0 = fine, else a KOALA_E_* code). */
 int koala_poll(koala_ctx *ctx, int *done, int *device_status);
@@ -289,10 +271,15 @@ int koala_gemm_bf16(const void *X, const void *X_lo /* optional residual of X, s
  * device's memory limit.  The split-K partial sums go to a fixed 8 MiB array inside the library's
  * device image (koala_gemm_static_scratch_bytes(); every GPU that loads the library holds it until
  * the process exits).  Nothing is allocated or freed on the device, by this call or under it.
- *   - split_k * M * N_out * 4 bytes must fit in the array, else KOALA_E_CAPACITY (split_k 0 =
- *     automatic; split_k 1 needs no scratch at all).  K_in % 64 == 0, X rows as koala_gemm_x_rows.
- *   - The first call on each device looks up the array's device address (with that device
- *     current) and prepares the kernel; make that first call outside any stream capture.
+ *   - split_k: 1..8 = that many partial sums per output, which must fit in the array
+ *     (split_k * M * N_out * 4 bytes <= 8 MiB, else KOALA_E_CAPACITY; split_k 1 needs no scratch at
+ *     all and is accepted at any size); 0 = automatic: the factor the multiply would choose by
+ *     itself, lowered until it fits (never an error for size); above 8: KOALA_E_INVALID.
+ *     K_in % 64 == 0, X rows as koala_gemm_x_rows.
+ *   - The first call on each device (with that device current) looks up the array's device address
+ *     and prepares the kernel for that device.  With CUDA's lazy module loading that look-up is also
+ *     the moment the 8 MiB get their device memory, so make this first call at start-up, before
+ *     memory is tight, and outside any stream capture.
  *   - All calls on a device share the one array and it keeps the previous call's contents (none of
  *     which is read before it is overwritten).  Two calls whose kernels may overlap on the GPU
  *     (different streams, no ordering between them) race on it: order them on one stream or with

@@ -20,7 +20,7 @@ ERR_NAMES = {0: "KOALA_OK", 1: "KOALA_E_INVALID", 2: "KOALA_E_UNSUPPORTED", 3: "
              4: "KOALA_E_STATE", 5: "KOALA_E_CUDA", 6: "KOALA_E_TIMEOUT"}
 KOALA_FP32, KOALA_BF16 = 0, 1
 KOALA_EAGLE, KOALA_MEDUSA = 0, 1
-KOALA_F_NO_TENSOR_CORES, KOALA_F_NO_PDL, KOALA_F_BF16_ACTIVATIONS = 1, 2, 4
+KOALA_F_NO_TENSOR_CORES, KOALA_F_NO_PDL = 1, 2
 LAYER_TENSORS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")
 
 
@@ -114,6 +114,10 @@ def load_library(rebuild: bool = False) -> C.CDLL:
     lib.koala_set_tuning.argtypes = [C.c_int, C.c_int]
     lib.koala_launch_count.restype = C.c_uint64
     lib.koala_launch_count.argtypes = []
+    lib.koala_selftest_timeout.restype = C.c_int
+    lib.koala_selftest_timeout.argtypes = [C.c_void_p, C.c_int]
+    lib.koala_debug_check_guards.restype = C.c_int
+    lib.koala_debug_check_guards.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     lib.koala_poll.restype = C.c_int
     lib.koala_poll.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     lib.koala_last_error.restype = C.c_char_p
@@ -313,6 +317,16 @@ class Koala:
 
     def launch_count(self) -> int:
         return int(self.lib.koala_launch_count())
+
+    def selftest_timeout(self, limit_cycles: int):
+        """Diagnostic: enqueues a one-thread kernel whose bounded wait runs out (see koala_debug.h)."""
+        self._check(self.lib.koala_selftest_timeout(self._ctx, int(limit_cycles)))
+
+    def check_guards(self):
+        """Diagnostic: (guards, damaged guards) of the workspace (synchronises the stream)."""
+        n, bad = C.c_int(0), C.c_int(0)
+        self._check(self.lib.koala_debug_check_guards(self._ctx, C.byref(n), C.byref(bad)))
+        return n.value, bad.value
 
     def poll(self):
         done, status = C.c_int(0), C.c_int(0)

@@ -380,13 +380,12 @@ size_t attn_mma_scratch_floats(int rows_total, int n_heads, int chunks) {
 cudaError_t tree_attention_mma(Launch L, const float *q, const void *k_cache, const void *v_cache,
                                RowPlan plan, Operand out, float *scratch, int rows_per_seq, int B,
                                int n_heads, int S_max, int chunks) {
-  static bool configured = false;
+  static SmemOptIn optin;
   const size_t smem = (size_t)NST * 2 * TILE_BYTES;
   static_assert((size_t)4 * 16 * MSTRIDE * sizeof(float) <= (size_t)NST * 2 * TILE_BYTES, "merge buffer fits");
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(tree_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  {
+    cudaError_t e = optin.ensure((const void *)tree_attn_mma_kernel, smem);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   const int rgs = (rows_per_seq + 15) / 16;
   if (rgs < 1 || rgs > 8 || chunks < 1) return cudaErrorInvalidValue;

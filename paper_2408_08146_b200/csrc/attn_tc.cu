@@ -131,7 +131,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   constexpr int NC = DUP ? 32 : 64;      // score columns (keys of a tile) per thread
   constexpr int ND = DUP ? 64 : 128;     // output dims per thread
   extern __shared__ unsigned char smem_raw[];
-  __shared__ uint64_t q_full, kv_full[NKV], kv_empty[NKV], s_full[2], p_full, o_full, x_bar[2];
+  __shared__ uint64_t q_full, kv_full[NKV], kv_empty[NKV], s_full[2], p_full, o_full, x_bar[2], drain_bar;
   __shared__ float xch[2][128];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int s_error;
@@ -152,6 +152,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     for (int s = 0; s < NKV; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
     mbar_init(&p_full, (uint32_t)n_arrive);
     mbar_init(&o_full, 1);
+    mbar_init(&drain_bar, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s_full[i], 1);
       mbar_init(&x_bar[i], 2);
@@ -330,6 +331,20 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       for (int c0 = 0; c0 < NC; c0 += 16) tmem_ld16(base + (uint32_t)c0, v + c0);
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
       const int key0 = (tile_lo + t) * TK;
+      if (kv_len - key0 < TK) {
+        // The last tile reaches past kv_len: those cache slots were never written and may hold
+        // anything, NaN bit patterns included, and 0 x NaN in P V would poison every row.  Zero
+        // the value rows from kv_len on (a row is 128 bytes of each 64-dim block; the swizzle
+        // only permutes inside the row).  The tile has landed: S, which this warp waited for, was
+        // issued after it.  Every row warp in use writes the same zeros.
+        const uint32_t vb = sb + OFF_KV + (t % NKV) * KV_STAGE + 2 * SUB;
+        for (int kr = kv_len - key0 + lane; kr < TK; kr += 32) {
+#pragma unroll
+          for (int blk = 0; blk < 2; ++blk)
+#pragma unroll
+            for (int q = 0; q < 8; ++q) st_shared_v4(vb + blk * SUB + kr * 128 + q * 16, 0u, 0u, 0u, 0u);
+        }
+      }
       uint64_t vis = ok_row ? tile_visibility(mk0, mk1, key0, ctx, kv_len) : 0ull;
       if (DUP) vis >>= 32 * half;
       float m_t = -INFINITY;
@@ -452,6 +467,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     }
   }
   if (warp == 5) {
+    if (failed) {      // MMAs issued before a wait ran out may still be running: no free under them
+      if (lane == 0) {
+        umma_commit(&drain_bar);
+        (void)mbar_wait(&drain_bar, 0);
+      }
+      __syncwarp();
+    }
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
   }
   if (threadIdx.x == 0 && failed && P.status) atomicMax(P.status, E_TIMEOUT);
@@ -479,15 +501,11 @@ bool attn_tc_supported(int rows_per_seq, int head_dim, int S_max) {
 cudaError_t tree_attention_tc(Launch L, Operand q_pair, int q_rows_alloc, const void *k_cache, const void *v_cache,
                               RowPlan plan, Operand out, int rows_per_seq, int B, int n_heads, int S_max, int chunks,
                               int *status) {
-  static bool configured = false;
+  static SmemOptIn optin_dup, optin_full;
   const size_t smem = (size_t)SMEM_BYTES + 1024;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(tree_attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  cudaError_t e = optin_dup.ensure((const void *)tree_attn_tc_kernel<true>, smem);
+  if (e == cudaSuccess) e = optin_full.ensure((const void *)tree_attn_tc_kernel<false>, smem);
+  if (e != cudaSuccess) return e;
   if (chunks != 1 && chunks != 2 && chunks != 4 && chunks != 8) return cudaErrorInvalidValue;
   if (q_pair.hi == nullptr || q_pair.lo == nullptr) return cudaErrorInvalidValue;
   const long long rows = (long long)B * n_heads * S_max;

@@ -5,6 +5,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <mutex>
+
 typedef __nv_bfloat16 bf16;
 
 namespace koala {
@@ -105,6 +107,25 @@ static inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block
   return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
+// A kernel's dynamic shared-memory limit is an attribute of the function on ONE device: raise it
+// once per device the library is used on (one object per kernel, kept by its launcher).
+struct SmemOptIn {
+  std::mutex mu;
+  size_t done[64] = {};
+  cudaError_t ensure(const void *fn, size_t smem) {
+    if (smem <= 48 * 1024) return cudaSuccess;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (smem <= done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) done[dev] = smem;
+    return e;
+  }
+};
+
 // ---------------------------------------------------------------------------------------------
 // launcher interface (one per kernel family); every launcher is asynchronous on `st`
 // ---------------------------------------------------------------------------------------------
@@ -195,6 +216,9 @@ int tc_default_split(int n_tiles, int kblocks, int tokens);
 cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in, int R,
                     float *Y, int ldy, int split, size_t split_stride, int *status, int max_slots,
                     SplitIn *out);
+
+// selftest.cu : a wait that runs out on purpose, with nothing else in flight
+cudaError_t selftest_timeout(Launch L, int *status, long long limit_cycles);
 
 // tree.cu
 struct TreeBufs {

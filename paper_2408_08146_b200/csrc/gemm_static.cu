@@ -9,6 +9,8 @@
 #include "../../include/koala.h"
 #include "common.cuh"
 
+#include <mutex>
+
 namespace {
 
 // 8 MiB of fp32 partial sums; every device that loads the library holds this until the process exits.
@@ -16,7 +18,9 @@ constexpr size_t STATIC_SCRATCH_FLOATS = (size_t)2 * 1024 * 1024;
 static __device__ __align__(256) float g_static_scratch[STATIC_SCRATCH_FLOATS];
 
 constexpr int MAX_DEVICES = 64;
+constexpr int MAX_STATIC_SPLIT = 8;
 float *g_scratch_ptr[MAX_DEVICES] = {nullptr};   // device address of the array, per device
+std::mutex g_scratch_mu;
 
 }  // namespace
 
@@ -32,28 +36,41 @@ int koala_gemm_bf16_static(const void *X, const void *X_lo, const void *W, float
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return KOALA_E_CUDA;
   if (dev < 0 || dev >= MAX_DEVICES) return KOALA_E_UNSUPPORTED;
-  if (g_scratch_ptr[dev] == nullptr) {
-    // The array's name is only a host-side handle; kernels need its address on the current device.
-    float *p = nullptr;
-    if (cudaGetSymbolAddress((void **)&p, g_static_scratch) != cudaSuccess || p == nullptr) return KOALA_E_CUDA;
-    g_scratch_ptr[dev] = p;
+  if (split_k < 0 || split_k > MAX_STATIC_SPLIT) return KOALA_E_INVALID;
+  float *scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    if (g_scratch_ptr[dev] == nullptr) {
+      // The array's name is only a host-side handle; kernels need its address on the current device.
+      // (With lazy module loading this look-up is also what gives the array its device memory.)
+      float *p = nullptr;
+      if (cudaGetSymbolAddress((void **)&p, g_static_scratch) != cudaSuccess || p == nullptr) return KOALA_E_CUDA;
+      g_scratch_ptr[dev] = p;
+    }
+    scratch = g_scratch_ptr[dev];
   }
   char err[160];
-  if (tc_init_driver(err, sizeof(err)) != 0) return KOALA_E_CUDA;
+  if (tc_init_driver(err, sizeof(err)) != 0) return KOALA_E_CUDA;   // prepares this device once
   GemmMats m{{W, nullptr, nullptr}, {N_out, 0, 0}, 1};
   if (!tc_supported(m, K_in)) return KOALA_E_UNSUPPORTED;
-  int split = split_k > 0 ? split_k : tc_default_split((N_out + 127) / 128, K_in / 64, M);
+  const size_t stride = (size_t)M * N_out;
+  int split = split_k;
+  if (split == 0) {
+    // automatic: the factor the GEMM would choose, lowered until its partial sums fit in the array
+    // (a caller that cannot allocate has no other entry point to fall back to)
+    split = tc_default_split((N_out + 127) / 128, K_in / 64, M);
+    if (split > MAX_STATIC_SPLIT) split = MAX_STATIC_SPLIT;
+    const size_t fit = STATIC_SCRATCH_FLOATS / stride;
+    if ((size_t)split > fit) split = fit < 1 ? 1 : (int)fit;
+  }
   if (split > K_in / 64) split = K_in / 64;
-  if (split > 8) split = 8;
   Launch L{(cudaStream_t)cuda_stream, false};
   Operand Xo{const_cast<void *>(X), const_cast<void *>(X_lo)};
   const int rows_alloc = koala_gemm_x_rows(M, X_lo != nullptr);
   if (split == 1)
     return gemm_tc(L, Xo, rows_alloc, m, K_in, M, Y, ldy, 1, 0, device_status, 1, nullptr) == cudaSuccess ? KOALA_OK
                                                                                               : KOALA_E_CUDA;
-  const size_t stride = (size_t)M * N_out;
-  if ((size_t)split * stride > STATIC_SCRATCH_FLOATS) return KOALA_E_CAPACITY;
-  float *scratch = g_scratch_ptr[dev];
+  if ((size_t)split * stride > STATIC_SCRATCH_FLOATS) return KOALA_E_CAPACITY;   // an explicit factor that does not fit
   // every partial element that is read below is written by exactly one CTA of this launch, so the
   // previous call's contents need no clearing
   SplitIn s;

@@ -85,6 +85,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   __shared__ uint64_t empty_bar[MAX_STAGES];
   __shared__ uint64_t acc_full[2];      // accumulator buffer complete (MMA -> epilogue)
   __shared__ uint64_t acc_empty[2];     // accumulator buffer drained (epilogue -> MMA)
+  __shared__ uint64_t drain_bar;        // error path: every MMA issued so far has finished
   __shared__ uint32_t tmem_base_slot;
   __shared__ int s_error;
 
@@ -135,6 +136,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       mbar_init(&acc_full[i], 1);
       mbar_init(&acc_empty[i], 4);       // one arrival per epilogue warp
     }
+    mbar_init(&drain_bar, 1);
     s_error = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -316,6 +318,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
+    if (s_error) {
+      // a wait ran out somewhere in the block: MMAs issued before that may still be running, and
+      // tensor memory must not be freed under them
+      if (lane == 0) {
+        umma_commit(&drain_bar);
+        (void)mbar_wait(&drain_bar, 0);
+      }
+      __syncwarp();
+    }
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                  ::"r"(tmem_acc), "r"((uint32_t)(P.tmem_cols * P.nbuf * (P.wide ? 2 : 1)))
                  : "memory");
@@ -331,8 +342,25 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 EncodeTiledFn g_encode = nullptr;
 std::mutex g_mu;
 std::map<std::tuple<const void *, int, int, int>, CUtensorMap> g_maps;   // (ptr, rows, K, box rows)
-int g_smem_optin = 0;
-int g_num_sms = 148;
+// Per-device facts and set-up: the kernel's shared-memory opt-in is an attribute of the function on
+// one device, so every device the library is used on is prepared once (under g_mu).
+constexpr int MAX_DEVICES = 64;
+struct DevInfo {
+  bool ready;
+  int smem_optin, num_sms;
+};
+DevInfo g_dev[MAX_DEVICES] = {};
+thread_local int t_dev = 0;          // the calling thread's current device as of its last use_current_device()
+// Points the per-device facts at the calling thread's current device; false if that device was
+// never prepared by tc_init_driver().
+bool use_current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES || !g_dev[dev].ready) return false;
+  t_dev = dev;
+  return true;
+}
+#define g_smem_optin (g_dev[t_dev].smem_optin)
+#define g_num_sms (g_dev[t_dev].num_sms)
 int g_tune_stages = 0;      // 0 = as many as fit (at most 8)
 int g_tune_max_split = 0;   // 0 = default rule
 int g_tune_no_streamk = 0;  // 1 = always the per-tile decomposition
@@ -371,28 +399,40 @@ bool get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out
 bool tc_get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out) {
   return get_map(ptr, rows, K_in, box_rows, out);
 }
-int tc_smem_optin() { return g_smem_optin; }
+int tc_smem_optin() { return use_current_device() ? g_smem_optin : 0; }
 
+// Prepares the calling thread's current device (once per device) and remembers it for the
+// launchers that follow on this thread.
 int tc_init_driver(char *err, size_t errlen) {
-  std::lock_guard<std::mutex> lock(g_mu);
-  if (g_encode) return 0;
-  void *fn = nullptr;
-  cudaDriverEntryPointQueryResult q;
-  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
-  if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || fn == nullptr) {
-    snprintf(err, errlen, "cuTensorMapEncodeTiled not available: %s", cudaGetErrorString(e));
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) {
+    snprintf(err, errlen, "no usable current device: %s", cudaGetErrorString(e));
     return 1;
   }
-  int dev = 0;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&g_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-  e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g_smem_optin - 1024);
+  std::lock_guard<std::mutex> lock(g_mu);
+  t_dev = dev;
+  if (g_dev[dev].ready) return 0;
+  if (!g_encode) {
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || fn == nullptr) {
+      snprintf(err, errlen, "cuTensorMapEncodeTiled not available: %s", cudaGetErrorString(e));
+      return 1;
+    }
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  DevInfo d{};
+  cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, dev);
+  e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin - 1024);
   if (e != cudaSuccess) {
     snprintf(err, errlen, "cannot raise the GEMM kernel's shared memory: %s", cudaGetErrorString(e));
     return 1;
   }
-  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  d.ready = true;
+  g_dev[dev] = d;
   return 0;
 }
 
@@ -436,6 +476,7 @@ static int split_cap(int kblocks, int tokens) {
 }
 
 int tc_default_split(int n_tiles, int kblocks, int tokens) {
+  if (!use_current_device()) return 1;
   const int slots = 2 * g_num_sms;
   int s = slots / (n_tiles > 0 ? n_tiles : 1);
   const int cap = split_cap(kblocks, tokens);
@@ -488,6 +529,7 @@ int tc_streamk_ctas(int n_tiles, int kblocks, int tokens, int max_slots, int *sl
 cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in, int R,
                     float *Y, int ldy, int split, size_t split_stride, int *status, int max_slots,
                     SplitIn *out) {
+  if (!use_current_device()) return cudaErrorInitializationError;
   if (!tc_supported(m, K_in) || R < 1 || ((uintptr_t)X.hi & 15u) || ((uintptr_t)X.lo & 15u))
     return cudaErrorInvalidValue;
   TcParams P;

@@ -8,6 +8,7 @@
 
 #include "../../include/koala.h"
 #include "common.cuh"
+#include "koala_debug.h"
 
 using namespace koala;
 
@@ -27,14 +28,21 @@ struct LayerW {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Walks the workspace; with base == nullptr it only measures.
+constexpr size_t GUARD_BYTES = 256;
+constexpr int GUARD_PATTERN = 0xC5;
+
+// Walks the workspace; with base == nullptr it only measures.  Every buffer is followed by a guard
+// of GUARD_BYTES that nothing writes after koala_init (koala_debug_check_guards).
 struct Carver {
   unsigned char *base;
   size_t off;
+  std::vector<size_t> *guards;
   template <typename T> T *take(size_t count) {
     off = align_up(off, 256);
     T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
-    off += count * sizeof(T);
+    off = align_up(off + count * sizeof(T), 256);
+    if (guards) guards->push_back(off);
+    off += GUARD_BYTES;
     return p;
   }
 };
@@ -87,6 +95,8 @@ struct koala_ctx {
   size_t ev_used;                       // pairs in use
   uint64_t t_bytes[3];
   int32_t t_launches[3];
+  unsigned char *ws_base;
+  std::vector<size_t> guards;    // offsets of the guard words in the workspace
   char err[256];
 };
 
@@ -141,7 +151,8 @@ bool config_ok(const koala_config *cfg, char *why, size_t n) {
 
 // Assigns (or measures) every workspace buffer.  Must visit the same sequence in both modes.
 size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
-  Carver w{base, 0};
+  c->guards.clear();
+  Carver w{base, 0, base ? &c->guards : nullptr};
   const int B = cfg.B, N = cfg.N, H = cfg.H, F = cfg.F, V = cfg.V, k = cfg.topk;
   const int M = B * N;
   int draft_rows = B * k;
@@ -162,7 +173,7 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
   c->feat[0] = w.take<float>((size_t)(B * k + 16) * H);
   c->feat[1] = w.take<float>((size_t)(B * k + 16) * H);
   c->mx = w.take<float>((size_t)Mp * H);
-  const bool pair = cfg.dtype == KOALA_BF16 && (cfg.flags & KOALA_F_BF16_ACTIVATIONS) == 0;
+  const bool pair = cfg.dtype == KOALA_BF16;     // bf16 operands as value + rounding residual
   c->pair = pair;
   auto operand = [&](size_t cols) {
     Operand o;
@@ -558,6 +569,8 @@ int koala_init(const koala_config *cfg, const koala_weights *w, const koala_stat
     char e[160];
     if (tc_init_driver(e, sizeof(e)) != 0) return fail(c, KOALA_E_CUDA, "%s", e);
   }
+  c->ws_base = (unsigned char *)st->workspace;
+  for (size_t off : c->guards) CU_TRY(cudaMemsetAsync(c->ws_base + off, GUARD_PATTERN, GUARD_BYTES, c->st));
   // small state that must start at zero
   CU_TRY(cudaMemsetAsync(c->status, 0, 4 * sizeof(int), c->st));
   CU_TRY(cudaMemsetAsync(c->t.alpha_hits, 0, 128 * sizeof(unsigned long long), c->st));
@@ -650,7 +663,10 @@ int koala_verify(koala_ctx *c, const koala_tree *tree) {
     c->last_tree_from_caller = false;
     c->pend_cap = g.N < g.D + 1 ? g.N : g.D + 1;
   }
-  const int R = g.B * g.N;
+  // a single sequence with a short caller tree (a prompt chunk, a one-node step) runs n_max rows;
+  // with several sequences row b * N + u is fixed, so all B * N rows run
+  const int rows = (tree && g.B == 1) ? tree->n_max : g.N;
+  const int R = g.B == 1 ? rows : g.B * g.N;
   c->pending = RowScale{nullptr, 0, 0.f, 0.f};
   CU_TRY(tree_ancestors(LN(c), c->t, g.B, g.N));
   CU_TRY(plan_verify(LN(c), c->t, c->p, c->seq_len, g.B, g.N, g.head_dim, g.rope_base, g.S_max, c->status));
@@ -666,7 +682,7 @@ int koala_verify(koala_ctx *c, const koala_tree *tree) {
   const size_t le = kv_layer_elems(g) * c->esz;
   for (int l = 0; l < g.L; ++l) {
     const bool last = l == g.L - 1;
-    K_TRY(run_layer(c, c->layers[l], (unsigned char *)c->tk + l * le, (unsigned char *)c->tv + l * le, R, g.N,
+    K_TRY(run_layer(c, c->layers[l], (unsigned char *)c->tk + l * le, (unsigned char *)c->tv + l * le, R, rows,
                     last ? c->final_norm : c->layers[l + 1].attn_norm, last ? c->lmin : c->xn,
                     last ? c->verify_hid : nullptr, !last));
   }
@@ -795,6 +811,29 @@ int koala_timing_read(koala_ctx *c, koala_timing *out) {
 void koala_set_tuning(int key, int value) { koala::tc_set_tuning(key, value); }
 
 uint64_t koala_launch_count(void) { return (uint64_t)koala::g_launches; }
+
+int koala_selftest_timeout(koala_ctx *c, int limit_cycles) {
+  if (!c) return KOALA_E_INVALID;
+  if (limit_cycles < 1 || limit_cycles > 100000000) return fail(c, KOALA_E_INVALID, "limit_cycles outside 1..1e8");
+  CU_TRY(koala::selftest_timeout(LN(c), c->status, (long long)limit_cycles));
+  return KOALA_OK;
+}
+
+int koala_debug_check_guards(koala_ctx *c, int *n_guards, int *n_damaged) {
+  if (!c || !n_guards || !n_damaged) return KOALA_E_INVALID;
+  CU_TRY(cudaStreamSynchronize(c->st));
+  std::vector<unsigned char> host(GUARD_BYTES);
+  int bad = 0;
+  for (size_t off : c->guards) {
+    CU_TRY(cudaMemcpy(host.data(), c->ws_base + off, GUARD_BYTES, cudaMemcpyDeviceToHost));
+    bool same = true;
+    for (unsigned char v : host) same = same && v == (unsigned char)GUARD_PATTERN;
+    bad += same ? 0 : 1;
+  }
+  *n_guards = (int)c->guards.size();
+  *n_damaged = bad;
+  return KOALA_OK;
+}
 
 int koala_poll(koala_ctx *c, int *done, int *device_status) {
   if (!c) return KOALA_E_INVALID;

@@ -971,12 +971,10 @@ cudaError_t topk_logp(Launch L, const float *logits, int32_t *tok, float *logp, 
   if (V <= 32768 && k <= 32)
     return launch_k(topk_logp_fast_kernel, dim3(R), dim3(1024), 0, L.st, L.pdl, logits, tok, logp, V, k);
   const size_t smem = (size_t)V * sizeof(float);
-  static size_t configured = 0;
-  if (smem > 48 * 1024 && smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(topk_logp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+  static SmemOptIn optin;
+  {
+    cudaError_t e = optin.ensure((const void *)topk_logp_kernel, smem);
     if (e != cudaSuccess) return e;
-    configured = smem;
   }
   return launch_k(topk_logp_kernel, dim3(R), dim3(1024), smem, L.st, L.pdl, logits, tok, logp, V, k);
 }

@@ -217,22 +217,13 @@ accept_sampled_kernel(TreeBufs t, const float *verify_logits, const float *hid, 
   }
 }
 
-cudaError_t ensure_smem(const void *fn, size_t smem, size_t *configured) {
-  if (smem > 48 * 1024 && smem > *configured) {
-    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    *configured = smem;
-  }
-  return cudaSuccess;
-}
-
 }  // namespace
 
 cudaError_t sample_rows(Launch L, const float *logits, const float *u, int u_stride, int u_off, int32_t *tok,
                         float *logp, float *probs, int R, int V) {
-  static size_t configured = 0;
+  static SmemOptIn optin;
   const size_t smem = (size_t)V * sizeof(float);
-  cudaError_t e = ensure_smem((const void *)sample_rows_kernel, smem, &configured);
+  cudaError_t e = optin.ensure((const void *)sample_rows_kernel, smem);
   if (e != cudaSuccess) return e;
   return launch_k(sample_rows_kernel, dim3(R), dim3(NT), smem, L.st, L.pdl, logits, u, u_stride, u_off, tok, logp,
                   probs, V);
@@ -242,9 +233,9 @@ cudaError_t accept_sampled(Launch L, TreeBufs t, const float *verify_logits, con
                            const float *chain_d, const float *u_accept, const float *u_bonus, int32_t *seq_len,
                            int32_t *out_tokens, int out_stride, int32_t *out_len, int B, int N, int H, int V, int D,
                            int *status) {
-  static size_t configured = 0;
+  static SmemOptIn optin;
   const size_t smem = (size_t)V * sizeof(float);
-  cudaError_t e = ensure_smem((const void *)accept_sampled_kernel, smem, &configured);
+  cudaError_t e = optin.ensure((const void *)accept_sampled_kernel, smem);
   if (e != cudaSuccess) return e;
   return launch_k(accept_sampled_kernel, dim3(B), dim3(NT), smem, L.st, L.pdl, t, verify_logits, verify_hid, chain_d,
                   u_accept, u_bonus, seq_len, out_tokens, out_stride, out_len, N, H, V, D, status);

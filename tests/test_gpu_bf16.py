@@ -176,6 +176,18 @@ def test_t7_eagle_draft_and_verify(K):
     _teacher_forced_iteration(reduced(T7_EAGLE, 2, K=K))
 
 
+def test_t7_eagle_full_depth():
+    """The 7B configuration with the EAGLE-style head at full depth: 32 target layers, K = 2,
+    dynamic tree of 60 nodes, context 1024."""
+    _teacher_forced_iteration(T7_EAGLE)
+
+
+def test_t13_eagle_full_depth_batch4_ragged():
+    """The 13B configuration at full depth: 40 target layers, batch 4 with ragged contexts in
+    [512, 2048], 64-node trees (256 rows per forward)."""
+    _teacher_forced_iteration(T13_EAGLE)
+
+
 def test_t7_eagle_cuda_core_path_agrees():
     _teacher_forced_iteration(reduced(T7_EAGLE, 1, K=1, S_max=384, prompt_len=256), flags=1)
 

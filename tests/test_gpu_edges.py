@@ -126,6 +126,22 @@ def test_long_context_many_key_tiles_and_chunks(context):
 def test_tensor_core_attention_shapes(N, B, n_heads, context, S_max):
     """One bf16 layer with head_dim 128 at row counts, batch sizes and chunk counts that select
     every variant of the tcgen05 attention kernel; the tree sits on top of a random cache."""
+    _attention_case(N, B, n_heads, context, S_max)
+
+
+@pytest.mark.parametrize("N,B,n_heads,context,S_max", [
+    (60, 1, 32, 500, 1024),      # tcgen05 kernel, duplicated rows; the last key tile is partial
+    (100, 2, 32, 700, 1024),     # tcgen05 kernel, more than 64 rows
+    (8, 1, 32, 300, 512),        # fewer than 16 rows: the mma.sync kernel
+])
+def test_unwritten_cache_slots_may_hold_nan(N, B, n_heads, context, S_max):
+    """Only the slots below seq_len (and the tree's own) ever hold data the caller or the library
+    wrote; everything beyond may be uninitialised memory.  The slots from S + N on are filled with
+    NaN bit patterns here (plain data, nothing faults) and the result must not change."""
+    _attention_case(N, B, n_heads, context, S_max, poison=True)
+
+
+def _attention_case(N, B, n_heads, context, S_max, poison=False):
     H = n_heads * 128
     cfg = reduced(T7_EAGLE, 1, K=1, N=N, B=B, H=H, n_heads=n_heads, F=2 * H, V=2048, D=min(5, N - 1),
                   S_max=S_max, prompt_len=context)
@@ -138,6 +154,10 @@ def test_tensor_core_attention_shapes(N, B, n_heads, context, S_max):
         orc.target_v[0][b][...] = kv_to_oracle(eng.target_v, 0, b, np.float32)
         orc.seq_len[b] = lens[b]
     eng.seq_len.copy_(torch.tensor(lens, dtype=torch.int32))
+    if poison:
+        for b in range(B):
+            eng.target_k[:, b, :, lens[b] + N:, :] = float("nan")
+            eng.target_v[:, b, :, lens[b] + N:, :] = float("nan")
     par = [-1] + [max(0, u - 1 - (u * 7) % min(u, 5)) for u in range(1, N)]
     toks = [uniform_ints(11 + b, "edge.shapes", N, 0, cfg.V) for b in range(B)]
     eng.koala_verify(_tree_arrays(eng, toks, [par] * B))

@@ -103,3 +103,55 @@ def test_tree_helpers():
     assert vis[2].tolist() == [True, False, True, False, False]
     with pytest.raises(AssertionError):
         tree_levels([-1, 2, 0])
+
+
+def test_cache_storage_rounding_is_applied_to_rotated_keys_and_values_only(hw):
+    """Where the oracle rounds for a bf16 cache (the paper states no precision, Section 4.1; the
+    reading is: a key / value is rounded when it is written to the cache, after the rotary
+    embedding, and nothing else is rounded).
+
+    (1) A recording identity in place of the rounding: the run is bit-equal to the run without it,
+    it is called exactly twice per layer and forward, and what it is handed is exactly what the
+    un-rounded run stores (the rotated keys, the values) - so queries never pass through it and a
+    rounding placed before the rotation would be handed something else.
+    (2) With the real rounding, layer 0 (whose inputs do not depend on any cache) stores exactly
+    the rounded values of the un-rounded run, bit for bit, and later layers see a different cache.
+    """
+    from oracle.koala_oracle import round_to_bf16
+    toks = prompts(CFG)[0][:24]
+    par = np.arange(-1, len(toks) - 1)
+    plain = KoalaOracle(CFG, hw, dtype=np.float32)
+    ref_logits, _ = plain.target_forward(0, toks, par)
+
+    seen = []
+
+    def recording_identity(a):
+        seen.append(np.array(a, copy=True))
+        return a
+
+    rec = KoalaOracle(CFG, hw, dtype=np.float32, kv_round=recording_identity)
+    logits, _ = rec.target_forward(0, toks, par)
+    assert np.array_equal(logits, ref_logits)
+    assert len(seen) == 2 * CFG.L
+    n = len(toks)
+    for l in range(CFG.L):
+        assert seen[2 * l].shape == seen[2 * l + 1].shape == (n, CFG.n_heads, CFG.head_dim)
+        assert np.array_equal(seen[2 * l], plain.target_k[l][0][:n])        # rotated keys
+        assert np.array_equal(seen[2 * l + 1], plain.target_v[l][0][:n])    # values
+
+    rounded = KoalaOracle(CFG, hw, dtype=np.float32, kv_round=round_to_bf16)
+    r_logits, _ = rounded.target_forward(0, toks, par)
+    k0, v0 = rounded.target_k[0][0][:n], rounded.target_v[0][0][:n]
+    assert np.array_equal(k0.view(np.uint32), round_to_bf16(plain.target_k[0][0][:n]).view(np.uint32))
+    assert np.array_equal(v0.view(np.uint32), round_to_bf16(plain.target_v[0][0][:n]).view(np.uint32))
+    assert (k0.view(np.uint32) & 0xFFFF == 0).all() and (v0.view(np.uint32) & 0xFFFF == 0).all()
+    # rounding the keys before rotating them gives other bits: the check above can tell the two apart
+    from oracle.koala_oracle import rmsnorm, rope
+    x0 = hw("embed").astype(np.float32)[np.asarray(toks, dtype=np.int64)]
+    h0 = rmsnorm(x0, hw("layers.0.attn_norm").astype(np.float32), CFG.rms_eps)
+    k_pre = (h0 @ hw("layers.0.wk").astype(np.float32).T).reshape(n, CFG.n_heads, CFG.head_dim)
+    slip = rope(round_to_bf16(k_pre), np.arange(n), CFG.rope_base)
+    assert not np.array_equal(np.asarray(slip, np.float32).view(np.uint32), k0.view(np.uint32))
+    # the rounded cache changes the result, but only at the scale of bf16 rounding
+    d = np.abs(r_logits - ref_logits).max()
+    assert 0 < d < 5e-2

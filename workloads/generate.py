@@ -135,6 +135,12 @@ class WeightStore:
     def __getitem__(self, name: str) -> torch.Tensor:
         return self.tensors[name]
 
+    def to(self, device) -> "WeightStore":
+        """Moves every tensor (plain copies; the values were generated where the store was built)."""
+        self.device = torch.device(device)
+        self.tensors = {n: t.to(self.device) for n, t in self.tensors.items()}
+        return self
+
     def host(self, name: str, dtype=np.float64) -> np.ndarray:
         t = self.tensors[name]
         if dtype == np.float64:
