@@ -47,11 +47,29 @@ def test_single_rank_is_identity():
 
 
 def test_workload_capacity_and_bytes():
+    """Capacity rule and the algorithmic bytes / flops of a step, against numbers worked out by hand."""
     sys.path.insert(0, ROOT)
     import bench
-    cfg = bench.workload(100)
+    from workloads import T13_EAGLE, T7_EAGLE, T7_MEDUSA
+    cfg = bench.with_capacity(T7_MEDUSA, 100)
     assert cfg.S_max >= 512 + 100 * 5 + cfg.N and cfg.S_max % 128 == 0
-    ab = bench.algorithmic_bytes_per_step(cfg, 512.0)
-    assert ab["verify_weights"] == 32 * 202375168 * 2 + 32000 * 4096 * 2     # 7B layer matrices + LM head
+    ab = bench.algorithmic_work(cfg, 512.0)
+    layer7 = 202375168 * 2                                                    # 7B layer matrices, bf16
+    assert ab["verify_weights"] == 32 * layer7 + 32000 * 4096 * 2            # + LM head
     assert ab["draft_weights"] == 8 * 4096 * 4096 * 2 + 32000 * 4096 * 2
     assert ab["kv"] == 32 * 512 * 32 * 128 * 2 * 2
+    # EAGLE-style head, K = 2, 5 passes: fc + 2 layers + LM head per pass; the head's own cache per layer and pass
+    ab = bench.algorithmic_work(T7_EAGLE, 1024.0)
+    assert ab["draft_weights"] == 5 * (2 * 4096 * 4096 * 2 + 2 * layer7 + 32000 * 4096 * 2)
+    assert ab["kv"] == (32 + 5 * 2) * 1024 * 4096 * 2 * 2
+    # flops: 2 per weight and row; verify rows = B x N, draft rows = B x (1 + 4 x 10)
+    ab = bench.algorithmic_work(T13_EAGLE, 1280.0)
+    layer13 = (4 * 5120 * 5120 + 3 * 5120 * 13824) * 2
+    vw = 40 * layer13 + 32000 * 5120 * 2
+    pw = 2 * 5120 * 5120 * 2 + 2 * layer13 + 32000 * 5120 * 2
+    assert ab["verify_weights"] == vw
+    assert ab["flops"] == 2.0 * (vw / 2) * 256 + 2.0 * (pw / 2) * 4 * 41
+    peaks = {"hbm_gbs": 6400.0, "bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0, "source": "test"}
+    sr = bench.step_roofline(T13_EAGLE, 1280.0, 20.0, peaks)
+    assert sr["bound"] in ("hbm", "tensor") and 0 < sr["frac_of_peak"] < 1
+    assert abs(sr["frac_of_peak"] - max(sr["ideal_ms_hbm"], sr["ideal_ms_tensor"]) / 20.0) < 1e-12
