@@ -56,6 +56,10 @@ extern "C" {
 /* flags */
 #define KOALA_F_NO_TENSOR_CORES 1u /* run every GEMM on the CUDA-core path (debugging / A-B checks) */
 #define KOALA_F_NO_PDL 2u          /* launch kernels without programmatic dependent launch         */
+#define KOALA_F_LAYER_KERNEL 4u    /* run each decoder layer's matrix multiplies and the row-wise steps
+                                      between them in one persistent launch where that applies (bf16,
+                                      at most 128 rows per forward) instead of one kernel per step;
+                                      same results up to summation order, measured slower on B200    */
 
 #define KOALA_MAX_TREE 128 /* largest N: ancestor sets are 128-bit masks */
 #define KOALA_MAX_TOPK 16

@@ -20,7 +20,7 @@ ERR_NAMES = {0: "KOALA_OK", 1: "KOALA_E_INVALID", 2: "KOALA_E_UNSUPPORTED", 3: "
              4: "KOALA_E_STATE", 5: "KOALA_E_CUDA", 6: "KOALA_E_TIMEOUT"}
 KOALA_FP32, KOALA_BF16 = 0, 1
 KOALA_EAGLE, KOALA_MEDUSA = 0, 1
-KOALA_F_NO_TENSOR_CORES, KOALA_F_NO_PDL = 1, 2
+KOALA_F_NO_TENSOR_CORES, KOALA_F_NO_PDL, KOALA_F_LAYER_KERNEL = 1, 2, 4
 LAYER_TENSORS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")
 
 

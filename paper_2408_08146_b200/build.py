@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkoala.so")
-SOURCES = ["ops.cu", "gemm_simt.cu", "gemm_tc.cu", "attn_mma.cu", "attn_tc.cu", "tree.cu", "sampling.cu", "koala_api.cu", "gemm_static.cu", "selftest.cu"]
+SOURCES = ["ops.cu", "gemm_simt.cu", "gemm_tc.cu", "layer_tc.cu", "attn_mma.cu", "attn_tc.cu", "tree.cu", "sampling.cu", "koala_api.cu", "gemm_static.cu", "selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

@@ -485,12 +485,25 @@ int g_attn_tc_min_rows = 16;   // fewer query rows per sequence than this: the m
 
 void attn_tc_set_min_rows(int rows) { g_attn_tc_min_rows = rows; }
 
-// Key chunks (= cluster size) per (sequence, head): a power of two that keeps the CTA count within
-// the SMs, at most 8, with at least 128 keys of capacity per chunk.
+// Key chunks (= cluster size) per (sequence, head): 1, 2, 4 or 8, each chunk with at least 128 keys of
+// capacity.  One CTA per SM is resident, so `chunks * B * n_heads` CTAs run in rounds over the SMs; a
+// CTA costs a fixed part (set-up, the queries, the merge) plus its share of the key tiles.  The
+// estimate below, in microseconds from this kernel's measured tile and launch times, picks the
+// count with the shortest total (few sequences and heads: as many chunks as fill the SMs once;
+// more CTAs than SMs: shorter CTAs so that the last, partly filled round costs less).
 int attn_tc_chunks(int B, int n_heads, int S_max, int num_sms) {
-  int c = 1;
-  while (c < 8 && 2 * c * B * n_heads <= num_sms && 2 * c * 128 <= S_max) c *= 2;
-  return c;
+  const double fixed_us = 5.0, tile_us = 1.4;
+  const double tiles = (double)((S_max + TK - 1) / TK);
+  int best = 1;
+  double best_t = 0.0;
+  for (int c = 1; c <= 8; c *= 2) {
+    if (c > 1 && c * 128 > S_max) break;
+    const long long ctas = (long long)c * B * n_heads;
+    const double rounds = (double)((ctas + num_sms - 1) / num_sms);
+    const double t = rounds * (fixed_us + tile_us * tiles / c);
+    if (c == 1 || t < best_t - 1e-9) { best = c; best_t = t; }
+  }
+  return best;
 }
 
 bool attn_tc_supported(int rows_per_seq, int head_dim, int S_max) {

@@ -217,6 +217,42 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
                     float *Y, int ldy, int split, size_t split_stride, int *status, int max_slots,
                     SplitIn *out);
 
+// layer_tc.cu : several GEMMs of a decoder layer and the row-wise steps between them in one
+// persistent launch (bf16, activations as pairs, at most 128 rows, head_dim 128 for the rotary step)
+constexpr int LAYER_MAX_PHASES = 4;
+constexpr int LAYER_SYNC_WORDS = 2 * LAYER_MAX_PHASES + 1;   // done[], ready[] counters and the abort word
+enum { LAYER_POST_NONE = 0, LAYER_POST_ROW_UPDATE = 1, LAYER_POST_SWIGLU = 2, LAYER_POST_ROPE_KV = 3 };
+struct LayerPhaseJob {
+  Operand X;              // [x_rows_alloc][K_in] pair
+  int K_in;
+  GemmMats m;             // every n_out a multiple of 128
+  float *Y;               // partial sums: max_slots matrices split_stride floats apart, row stride ldy
+  int ldy;
+  size_t split_stride;
+  int max_slots;
+  int post;               // what consumes the partial sums
+  RowScale sc;            // SwiGLU / rotary step: RMSNorm scale still owed by this GEMM's input
+  const void *gain;       // residual update: gain of the norm that follows
+  Operand out;            // residual update: x * gain [R][ncols]; SwiGLU: activations [R][ncols]; rotary: query pair
+  float *sumsq;           // residual update: [R][ceil(ncols / 512)]
+  int ncols;              // residual update: H; SwiGLU: F
+};
+struct LayerJob {
+  LayerPhaseJob ph[LAYER_MAX_PHASES];
+  int n_phases;
+  int R, x_rows_alloc;
+  float *x;               // residual stream [R][H]
+  RowPlan plan;           // rotary step
+  float *q_out;
+  void *k_cache, *v_cache;
+  int rows_per_seq, n_heads, head_dim, S_max;
+};
+bool layer_stream_supported(const LayerJob &job);
+// sync: LAYER_SYNC_WORDS device words, zero at context start; use_count: host counters [LAYER_MAX_PHASES]
+// outs (optional): how each phase's partial sums are laid out, for a consumer outside the launch
+cudaError_t layer_stream(Launch L, const LayerJob &job, unsigned *sync, unsigned *use_count, int *status,
+                         SplitIn *outs);
+
 // selftest.cu : a wait that runs out on purpose, with nothing else in flight
 cudaError_t selftest_timeout(Launch L, int *status, long long limit_cycles);
 

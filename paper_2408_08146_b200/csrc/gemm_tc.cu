@@ -400,6 +400,7 @@ bool tc_get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *
   return get_map(ptr, rows, K_in, box_rows, out);
 }
 int tc_smem_optin() { return use_current_device() ? g_smem_optin : 0; }
+int tc_num_sms() { return use_current_device() ? g_num_sms : 0; }
 
 // Prepares the calling thread's current device (once per device) and remembers it for the
 // launchers that follow on this thread.

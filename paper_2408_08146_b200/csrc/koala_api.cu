@@ -66,6 +66,9 @@ struct koala_ctx {
   // workspace
   float *attn_part;
   float *sumsq[2];        // per-row partial sums of squares of the two deferred RMSNorms of a layer
+  unsigned *layer_sync;   // device counters of the persistent layer kernel
+  unsigned layer_use[LAYER_MAX_PHASES];   // how often each counter has been used (host)
+  bool stream_layers;     // decoder layers run through the persistent layer kernel where it applies
   RowScale pending;       // scale still owed by the consumer of the GEMM that reads c->xn
   int attn_chunks;
   float *x, *qbuf, *P, *verify_logits, *draft_logits, *verify_hid, *feat[2], *mx;
@@ -196,8 +199,9 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
   c->attn_part = (cfg.dtype == KOALA_BF16 && cfg.head_dim == 128)
                      ? w.take<float>(attn_mma_scratch_floats(Mp, cfg.n_heads, c->attn_chunks))
                      : nullptr;
-  c->sumsq[0] = w.take<float>((size_t)Mp * 8);
-  c->sumsq[1] = w.take<float>((size_t)Mp * 8);
+  c->sumsq[0] = w.take<float>((size_t)Mp * 32);
+  c->sumsq[1] = w.take<float>((size_t)Mp * 32);
+  c->layer_sync = w.take<unsigned>(LAYER_SYNC_WORDS);
   c->verify_tgt = w.take<int32_t>(Mp);
   c->s_parent = w.take<int32_t>(N);
   c->s_level = w.take<int32_t>(N);
@@ -244,6 +248,10 @@ size_t carve(koala_ctx *c, const koala_config &cfg, unsigned char *base) {
 }
 
 Launch LN(koala_ctx *c) { return Launch{c->st, c->pdl}; }
+
+size_t kv_layer_elems(const koala_config &g) {
+  return (size_t)g.B * g.n_heads * g.S_max * g.head_dim;
+}
 
 constexpr size_t MAX_TIMED = 8192;
 
@@ -304,6 +312,27 @@ int do_gemm(koala_ctx *c, Operand X, int K_in, GemmMats m, int R, float *direct,
     if (rc__ != KOALA_OK) return rc__; \
   } while (0)
 
+// Tree-masked attention of one layer over R rows: reads the rotated queries (fp32 and pair) and the
+// cache, writes the O projection's operand pair.
+int run_attention(koala_ctx *c, void *kc, void *vc, int R, int rows_per_seq) {
+  const koala_config &g = c->cfg;
+  const int ta = time_begin(c, KOALA_CLS_ATTENTION, 0);
+  if (c->use_tc && g.dtype == KOALA_BF16 && c->qpair.lo != nullptr &&
+      attn_tc_supported(rows_per_seq, g.head_dim, g.S_max)) {
+    CU_TRY(tree_attention_tc(LN(c), c->qpair, c->Mp, kc, vc, row_plan(c), c->attn_out, rows_per_seq, g.B, g.n_heads,
+                             g.S_max, attn_tc_chunks(g.B, g.n_heads, g.S_max, 148), c->status));
+  } else if (c->use_tc && g.head_dim == 128 && c->attn_part != nullptr && rows_per_seq <= 128) {
+    CU_TRY(tree_attention_mma(LN(c), c->qbuf, kc, vc, row_plan(c), c->attn_out, c->attn_part, rows_per_seq,
+                              g.B, g.n_heads, g.S_max,
+                              attn_mma_chunks(g.B, g.n_heads, rows_per_seq, g.S_max, 148)));
+  } else {
+    CU_TRY(tree_attention(LN(c), g.dtype, c->qbuf, kc, vc, row_plan(c), c->attn_out, R, rows_per_seq, g.B,
+                          g.n_heads, g.head_dim, g.S_max));
+  }
+  time_end(c, ta);
+  return KOALA_OK;
+}
+
 // One pre-norm decoder layer over R rows.  On entry x holds the residual stream and xn the
 // normalised input of the attention block.  On exit x is updated and `next_xn` holds
 // T(rmsnorm(x) * next_g) (or T(x) if next_g is null); `out_f32` optionally receives the same in fp32.
@@ -324,20 +353,7 @@ int run_layer(koala_ctx *c, const LayerW &w, void *kc, void *vc, int R, int rows
   CU_TRY(rope_kv_write(LN(c), g.dtype, s, c->pending, row_plan(c), c->qbuf, c->qpair, kc, vc, R, rows_per_seq, g.n_heads,
                        g.head_dim, g.S_max));
   c->pending = none;
-  const int ta = time_begin(c, KOALA_CLS_ATTENTION, 0);
-  if (c->use_tc && g.dtype == KOALA_BF16 && c->qpair.lo != nullptr &&
-      attn_tc_supported(rows_per_seq, g.head_dim, g.S_max)) {
-    CU_TRY(tree_attention_tc(LN(c), c->qpair, c->Mp, kc, vc, row_plan(c), c->attn_out, rows_per_seq, g.B, g.n_heads,
-                             g.S_max, attn_tc_chunks(g.B, g.n_heads, g.S_max, 148), c->status));
-  } else if (c->use_tc && g.head_dim == 128 && c->attn_part != nullptr && rows_per_seq <= 128) {
-    CU_TRY(tree_attention_mma(LN(c), c->qbuf, kc, vc, row_plan(c), c->attn_out, c->attn_part, rows_per_seq,
-                              g.B, g.n_heads, g.S_max,
-                              attn_mma_chunks(g.B, g.n_heads, rows_per_seq, g.S_max, 148)));
-  } else {
-    CU_TRY(tree_attention(LN(c), g.dtype, c->qbuf, kc, vc, row_plan(c), c->attn_out, R, rows_per_seq, g.B,
-                          g.n_heads, g.head_dim, g.S_max));
-  }
-  time_end(c, ta);
+  K_TRY(run_attention(c, kc, vc, R, rows_per_seq));
   GemmMats o{{w.wo, nullptr, nullptr}, {H, 0, 0}, 1};
   K_TRY(do_gemm(c, c->attn_out, H, o, R, nullptr, 0, &s));
   RowScale ffn = none;
@@ -361,8 +377,124 @@ int run_layer(koala_ctx *c, const LayerW &w, void *kc, void *vc, int R, int rows
   return KOALA_OK;
 }
 
-size_t kv_layer_elems(const koala_config &g) {
-  return (size_t)g.B * g.n_heads * g.S_max * g.head_dim;
+
+// n_layers pre-norm decoder layers over R rows.  On entry x holds the residual stream and c->xn the
+// first layer's input (normalised, or x * gain with its scale pending in c->pending).  After the
+// last layer the output is rmsnorm(x) * final_g (or x if final_g is null) as an operand in
+// `final_xn` and, optionally, in fp32 in `out_f32`.
+// Where the persistent layer kernel applies (bf16 pairs, at most 128 rows, head_dim 128, matrices
+// of whole 128-row tiles) a layer is two launches: attention, and one launch that runs
+// O -> residual -> gate/up -> SwiGLU -> down -> residual -> the next layer's Q/K/V -> rotary/cache.
+int run_layers(koala_ctx *c, const std::vector<LayerW> &layers, int n_layers, void *kbase, void *vbase, int R,
+               int rows_per_seq, const void *final_g, Operand final_xn, float *out_f32) {
+  const koala_config &g = c->cfg;
+  const int H = g.H, F = g.F;
+  const size_t le = kv_layer_elems(g) * c->esz;
+  auto kc_of = [&](int l) { return (void *)((unsigned char *)kbase + (size_t)l * le); };
+  auto vc_of = [&](int l) { return (void *)((unsigned char *)vbase + (size_t)l * le); };
+  bool streamed = c->stream_layers && g.dtype == KOALA_BF16 && c->pair && g.head_dim == 128 && R <= 128 &&
+                  c->qpair.lo != nullptr && n_layers > 0;
+  LayerJob job;
+  const size_t stride = (size_t)c->Mp * c->pcols;     // one partial-sum matrix of the widest GEMM
+  auto base_job = [&]() {
+    memset(&job, 0, sizeof(job));
+    job.R = R;
+    job.x_rows_alloc = c->Mp;
+    job.x = c->x;
+    job.plan = row_plan(c);
+    job.q_out = c->qbuf;
+    job.rows_per_seq = rows_per_seq;
+    job.n_heads = g.n_heads;
+    job.head_dim = g.head_dim;
+    job.S_max = g.S_max;
+  };
+  auto phase = [&](int i, Operand X, int K_in, GemmMats m, int post) -> LayerPhaseJob & {
+    LayerPhaseJob &j = job.ph[i];
+    int ncols = 0;
+    for (int q = 0; q < m.n; ++q) ncols += m.n_out[q];
+    j.X = X; j.K_in = K_in; j.m = m; j.Y = c->P; j.ldy = ncols; j.split_stride = (size_t)c->Mp * ncols;
+    j.max_slots = MAX_SPLIT; j.post = post;
+    j.sc = RowScale{nullptr, 0, 0.f, 0.f};
+    (void)stride;
+    return j;
+  };
+  const int chunks = (H + 511) / 512;
+  auto qkv_phase = [&](int i, const LayerW &w, RowScale sc) {
+    LayerPhaseJob &j = phase(i, c->xn, H, GemmMats{{w.wq, w.wk, w.wv}, {H, H, H}, 3}, LAYER_POST_ROPE_KV);
+    j.sc = sc;
+    j.out = c->qpair;
+  };
+  auto weight_bytes = [&](const LayerJob &jb) {
+    uint64_t b = 0;
+    for (int i = 0; i < jb.n_phases; ++i)
+      for (int q = 0; q < jb.ph[i].m.n; ++q) b += (uint64_t)jb.ph[i].m.n_out[q] * jb.ph[i].K_in * c->esz;
+    return b;
+  };
+  if (streamed) {
+    // dry run of the shapes: every launch of the sequence must be supported, else the per-kernel path
+    base_job();
+    qkv_phase(0, layers[0], c->pending);
+    job.k_cache = kc_of(0); job.v_cache = vc_of(0);
+    job.n_phases = 1;
+    streamed = layer_stream_supported(job);
+    if (streamed) {
+      LayerPhaseJob &a = phase(0, c->attn_out, H, GemmMats{{layers[0].wo, nullptr, nullptr}, {H, 0, 0}, 1}, LAYER_POST_ROW_UPDATE);
+      a.gain = layers[0].ffn_norm; a.out = c->xn; a.sumsq = c->sumsq[0]; a.ncols = H;
+      LayerPhaseJob &b = phase(1, c->xn, H, GemmMats{{layers[0].wg, layers[0].wu, nullptr}, {F, F, 0}, 2}, LAYER_POST_SWIGLU);
+      b.out = c->act; b.ncols = F;
+      phase(2, c->act, F, GemmMats{{layers[0].wd, nullptr, nullptr}, {H, 0, 0}, 1}, LAYER_POST_NONE);
+      job.n_phases = 3;
+      streamed = layer_stream_supported(job);
+    }
+  }
+  if (!streamed) {
+    for (int l = 0; l < n_layers; ++l) {
+      const bool last = l == n_layers - 1;
+      K_TRY(run_layer(c, layers[l], kc_of(l), vc_of(l), R, rows_per_seq, last ? final_g : layers[l + 1].attn_norm,
+                      last ? final_xn : c->xn, last ? out_f32 : nullptr, !last));
+    }
+    return KOALA_OK;
+  }
+  const RowScale none{nullptr, 0, 0.f, 0.f};
+  const RowScale ffn_scale{c->sumsq[0], chunks, 1.f / (float)H, g.rms_eps};
+  const RowScale attn_scale{c->sumsq[1], chunks, 1.f / (float)H, g.rms_eps};
+  // the first layer's Q/K/V with the rotary step
+  base_job();
+  qkv_phase(0, layers[0], c->pending);
+  job.k_cache = kc_of(0); job.v_cache = vc_of(0);
+  job.n_phases = 1;
+  {
+    const int tb = time_begin(c, KOALA_CLS_GEMM_TC, weight_bytes(job));
+    CU_TRY(layer_stream(LN(c), job, c->layer_sync, c->layer_use, c->status, nullptr));
+    time_end(c, tb);
+  }
+  c->pending = none;
+  for (int l = 0; l < n_layers; ++l) {
+    const bool last = l == n_layers - 1;
+    const LayerW &w = layers[l];
+    K_TRY(run_attention(c, kc_of(l), vc_of(l), R, rows_per_seq));
+    base_job();
+    LayerPhaseJob &a = phase(0, c->attn_out, H, GemmMats{{w.wo, nullptr, nullptr}, {H, 0, 0}, 1}, LAYER_POST_ROW_UPDATE);
+    a.gain = w.ffn_norm; a.out = c->xn; a.sumsq = c->sumsq[0]; a.ncols = H;
+    LayerPhaseJob &b = phase(1, c->xn, H, GemmMats{{w.wg, w.wu, nullptr}, {F, F, 0}, 2}, LAYER_POST_SWIGLU);
+    b.sc = ffn_scale; b.out = c->act; b.ncols = F;
+    LayerPhaseJob &d = phase(2, c->act, F, GemmMats{{w.wd, nullptr, nullptr}, {H, 0, 0}, 1},
+                             last ? LAYER_POST_NONE : LAYER_POST_ROW_UPDATE);
+    job.n_phases = 3;
+    if (!last) {
+      d.gain = layers[l + 1].attn_norm; d.out = c->xn; d.sumsq = c->sumsq[1]; d.ncols = H;
+      qkv_phase(3, layers[l + 1], attn_scale);
+      job.k_cache = kc_of(l + 1); job.v_cache = vc_of(l + 1);
+      job.n_phases = 4;
+    }
+    SplitIn outs[LAYER_MAX_PHASES];
+    const int tb = time_begin(c, KOALA_CLS_GEMM_TC, weight_bytes(job));
+    CU_TRY(layer_stream(LN(c), job, c->layer_sync, c->layer_use, c->status, outs));
+    time_end(c, tb);
+    if (last)
+      CU_TRY(row_epilogue(LN(c), g.dtype, 0, c->x, outs[2], nullptr, final_g, final_xn, out_f32, R, H, g.rms_eps));
+  }
+  return KOALA_OK;
 }
 
 int draft_eagle(koala_ctx *c, int pass) {
@@ -395,13 +527,7 @@ int draft_eagle(koala_ctx *c, int pass) {
   } else {
     CU_TRY(row_epilogue(LN(c), g.dtype, 1, c->x, s, c->fc_b, c->draft_layers[0].attn_norm, c->xn, nullptr,
                         R, H, g.rms_eps));
-    const size_t le = kv_layer_elems(g) * c->esz;
-    for (int j = 0; j < g.K; ++j) {
-      const bool last = j == g.K - 1;
-      K_TRY(run_layer(c, c->draft_layers[j], (unsigned char *)c->dk + j * le, (unsigned char *)c->dv + j * le,
-                      R, rows, last ? nullptr : c->draft_layers[j + 1].attn_norm, last ? lm_all : c->xn,
-                      last ? f_all : nullptr, !last));
-    }
+    K_TRY(run_layers(c, c->draft_layers, g.K, c->dk, c->dv, R, rows, nullptr, lm_all, f_all));
   }
   int lm_rows = R;
   if (pass == 0) {
@@ -573,6 +699,9 @@ int koala_init(const koala_config *cfg, const koala_weights *w, const koala_stat
   for (size_t off : c->guards) CU_TRY(cudaMemsetAsync(c->ws_base + off, GUARD_PATTERN, GUARD_BYTES, c->st));
   // small state that must start at zero
   CU_TRY(cudaMemsetAsync(c->status, 0, 4 * sizeof(int), c->st));
+  CU_TRY(cudaMemsetAsync(c->layer_sync, 0, LAYER_SYNC_WORDS * sizeof(unsigned), c->st));
+  memset(c->layer_use, 0, sizeof(c->layer_use));
+  c->stream_layers = c->use_tc && (g.flags & KOALA_F_LAYER_KERNEL) != 0;
   CU_TRY(cudaMemsetAsync(c->t.alpha_hits, 0, 128 * sizeof(unsigned long long), c->st));
   CU_TRY(cudaMemsetAsync(c->t.alpha_trials, 0, 128 * sizeof(unsigned long long), c->st));
   CU_TRY(cudaMemsetAsync(c->t.n_pend, 0, g.B * sizeof(int32_t), c->st));
@@ -679,13 +808,7 @@ int koala_verify(koala_ctx *c, const koala_tree *tree) {
     CU_TRY(embed_norm(LN(c), g.dtype, c->p.row_tok, c->embed, c->layers[0].attn_norm, c->x, c->xn, R, g.H, g.V,
                       g.rms_eps));
   }
-  const size_t le = kv_layer_elems(g) * c->esz;
-  for (int l = 0; l < g.L; ++l) {
-    const bool last = l == g.L - 1;
-    K_TRY(run_layer(c, c->layers[l], (unsigned char *)c->tk + l * le, (unsigned char *)c->tv + l * le, R, rows,
-                    last ? c->final_norm : c->layers[l + 1].attn_norm, last ? c->lmin : c->xn,
-                    last ? c->verify_hid : nullptr, !last));
-  }
+  K_TRY(run_layers(c, c->layers, g.L, c->tk, c->tv, R, rows, c->final_norm, c->lmin, c->verify_hid));
   GemmMats lm{{c->lm_head, nullptr, nullptr}, {g.V, 0, 0}, 1};
   K_TRY(do_gemm(c, c->lmin, g.H, lm, R, c->verify_logits, g.V, nullptr));
   CU_TRY(argmax_rows(LN(c), c->verify_logits, c->verify_tgt, R, g.V));

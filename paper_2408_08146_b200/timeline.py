@@ -37,7 +37,8 @@ def main():
     from workloads.generate import WeightStore, medusa_static_tree, prompts
     from . import Koala
 
-    cfg = bench.workload(100)
+    from workloads import T7_MEDUSA
+    cfg = bench.with_capacity(T7_MEDUSA, 100)
     store = WeightStore(cfg, "cuda:0")
     eng = Koala(cfg, store.tensors, static_tree=medusa_static_tree(cfg.N, cfg.n_medusa_heads, cfg.topk))
     eng.prefill(prompts(cfg), 64)
@@ -63,9 +64,9 @@ def main():
     print("critical-path increments per kernel name:")
     for k, (c, t) in sorted(inc.items(), key=lambda kv: -kv[1][1]):
         print(f"  {k:28s} n={c:4d}  sum {t:8.1f} us  avg {t / c:6.2f} us")
-    per_layer = [i for i, k in enumerate(seg) if "rope_kv" in k[2]]
+    per_layer = [i for i, k in enumerate(seg) if "tree_attn" in k[2]]      # one attention launch per decoder layer
     if len(per_layer) > args.layer + 1:
-        i0, i1 = per_layer[args.layer] - 1, per_layer[args.layer + 1] - 1
+        i0, i1 = per_layer[args.layer], per_layer[args.layer + 1]
         t0 = seg[i0][0]
         print(f"kernels of decoder layer {args.layer} (us from the layer's first kernel start):")
         for s, e, n in seg[i0:i1]:

@@ -188,6 +188,14 @@ def test_t13_eagle_full_depth_batch4_ragged():
     _teacher_forced_iteration(T13_EAGLE)
 
 
+@pytest.mark.parametrize("cfg", [reduced(T7_EAGLE, 3, K=2), reduced(T7_MEDUSA, 3), reduced(T13_EAGLE, 2, B=2)],
+                         ids=["t7_eagle", "t7_medusa", "t13_eagle_batch2"])
+def test_persistent_layer_kernel_path(cfg):
+    """KOALA_F_LAYER_KERNEL: the same iteration with each layer's matrix multiplies and row-wise
+    steps in one persistent launch (draft passes of 1..20 rows, verification of 60 / 64 / 128 rows)."""
+    _teacher_forced_iteration(cfg, flags=4)
+
+
 def test_t7_eagle_cuda_core_path_agrees():
     _teacher_forced_iteration(reduced(T7_EAGLE, 1, K=1, S_max=384, prompt_len=256), flags=1)
 

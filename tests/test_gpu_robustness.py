@@ -52,14 +52,14 @@ def _caller_tree(cfg, seed):
     return to(tok), to(np.tile(np.asarray(par), (B, 1))), to(np.full(B, N)), N
 
 
-@pytest.mark.parametrize("B,N", [(1, 60), (2, 64), (4, 64)])
-def test_same_forward_twice_is_bit_equal(B, N):
+@pytest.mark.parametrize("B,N,flags", [(1, 60, 0), (2, 64, 0), (4, 64, 0), (1, 60, 4), (2, 64, 4)])
+def test_same_forward_twice_is_bit_equal(B, N, flags):
     """The split-K, stream-K and 256-row-tile reductions add their partial sums in a fixed order:
     the same 7B-shaped verification (two layers; 60 rows: classic split-K and stream-K; 128 and
     256 rows: wide tiles and several token tiles) run twice gives identical bits."""
     cfg = reduced(T7_EAGLE, 2, K=1, B=B, N=N, S_max=768, prompt_len=512)
     store = WeightStore(cfg, DEV)
-    eng = Koala(cfg, store.tensors)
+    eng = Koala(cfg, store.tensors, flags=flags)     # flags 4: the persistent layer kernel's stream-K sums
     eng.target_k.copy_(random_kv(cfg, "target_k", cfg.L, DEV))
     eng.target_v.copy_(random_kv(cfg, "target_v", cfg.L, DEV))
     eng.seq_len.fill_(cfg.prompt_len)
