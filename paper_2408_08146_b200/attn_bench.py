@@ -36,10 +36,12 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--mma-sync", action="store_true")
+    ap.add_argument("--chunks", type=int, default=0, help="key chunks per (sequence, head): 1, 2, 4, 8; 0 = automatic")
     args = ap.parse_args()
     lib = binding.load_library()
     if args.mma_sync:
         lib.koala_set_tuning(9, 1 << 20)
+    lib.koala_set_tuning(12, args.chunks)
     n = args.rows
     cfg = reduced(T7_EAGLE, 2, K=1, N=n, B=args.batch, D=min(5, max(1, n - 1)), V=4096,
                   S_max=((args.context + n + 127) // 128) * 128)
@@ -58,7 +60,7 @@ def main():
     assert eng.device_status() == 0
     us = 1e3 * t["ms"] / t["launches"]
     kv = args.batch * cfg.n_heads * (args.context + n) * cfg.head_dim * 2 * 2
-    print(f"attention: rows {n} x batch {args.batch}, context {args.context}: {us:.2f} us per launch "
+    print(f"attention (chunks {args.chunks or 'auto'}): rows {n} x batch {args.batch}, context {args.context}: {us:.2f} us per launch "
           f"({t['launches']} launches, event-bracketed), {kv / 1e6:.2f} MB of K/V per launch = {kv / us / 1e3:.0f} GB/s")
     eng.close()
 

@@ -5,20 +5,23 @@
 //   S[128 x 64]  = Q K^T          tcgen05.mma, A = Q (K-major), B = K tile (K-major), fp32 in TMEM
 //   P            = exp2(S*c - m)  by the thread that owns the query row's TMEM lane: tcgen05.ld,
 //                                 mask, row max / sum without shuffles, P written to shared memory
-//   O_t[128x128] = P V            tcgen05.mma, A = P (K-major), B = V tile as stored, [key][dim],
-//                                 which is the MN-major operand form
-// and the rows fold O_t into their running (max, sum, O) in registers.  Q and P enter the MMAs as
-// bf16 pairs (value + rounding residual: two accumulating MMAs), so only the cached K and V carry
-// bf16 rounding.  Q (written as a pair by the rotary-embedding kernel) and the K/V tiles arrive by
-// TMA with the 128-byte swizzle, K/V in a two-stage ring; S is double-buffered in tensor memory, so
-// the tensor pipe computes the scores of tile t+1 while the rows process tile t.
+//   O[128x128]  += P V            tcgen05.mma, A = P (K-major), B = V tile as stored, [key][dim],
+//                                 which is the MN-major operand form; O stays in tensor memory
+// O accumulates over all tiles of the chunk.  A row's exponentials are relative to a reference
+// maximum that is raised only when a tile's maximum exceeds it by more than 2^8; only then is the
+// row's O rescaled in tensor memory (tcgen05.ld / st), so in the common case the rows never wait
+// for P V: the tensor pipe computes S of tile t+1 and P V of tile t-1 while the rows turn S of tile
+// t into P (two S buffers in tensor memory, two P buffers in shared memory).  Q and P enter the
+// MMAs as bf16 pairs (value + rounding residual: two accumulating MMAs), so only the cached K and V
+// carry bf16 rounding.  Q (written as a pair by the rotary-embedding kernel) and the K/V tiles
+// arrive by TMA with the 128-byte swizzle, K/V in a three-stage ring.
 // Warps 0..3 own the rows, warp 4 lane 0 issues the copies, warp 5 lane 0 the MMAs.
 // With several chunks the CTAs of one (head, sequence) form a thread-block cluster: every CTA
 // pushes, into each peer's shared memory, that peer's slice of the head dimension of its
 // unnormalised (O, m, l); after a cluster barrier every CTA merges its slice over the chunks in
-// chunk order from its own shared memory and writes it as a matrix-multiply operand pair.  (With
-// more than 64 rows the receive buffer reuses the K/V ring, so a first cluster barrier makes sure
-// that every peer is done with its tiles.)
+// chunk order from its own shared memory and writes it as a matrix-multiply operand pair.  (The
+// receive buffer reuses the K/V ring, so a first cluster barrier makes sure that every peer is done
+// with its tiles.)
 // The mask is: slots below ctx_len visible to every row; slot ctx_len + j visible to a row iff
 // bit j of its 128-bit mask; slots from kv_len on invisible.
 // Every wait is bounded: on expiry the kernel records a timeout in *status and returns.
@@ -29,30 +32,29 @@ namespace koala {
 
 bool tc_get_map(const void *ptr, int rows, int K_in, int box_rows, CUtensorMap *out);
 int tc_smem_optin();
+int tc_num_sms();
 
 namespace {
 
 constexpr int DH = 128;
 constexpr int TK = 64;                       // keys per tile
-constexpr int NKV = 2;                       // K/V stages
+constexpr int NKV = 3;                       // K/V stages
 constexpr int SUB = 64 * 64 * 2;             // one [64 keys][64 dims] block: 8 KB
 constexpr int QSUB = 128 * 64 * 2;           // one [128 rows][64 columns] block: 16 KB
 constexpr int OFF_Q = 0;                     // Q hi (2 blocks), Q lo (2 blocks)
 constexpr int OFF_KV = 4 * QSUB;             // stages of K (2 blocks) + V (2 blocks)
 constexpr int KV_STAGE = 4 * SUB;
-constexpr int OFF_P = OFF_KV + NKV * KV_STAGE;   // P hi, P lo
+constexpr int OFF_P = OFF_KV + NKV * KV_STAGE;   // two buffers of P hi, P lo
 constexpr int P_BUF = 2 * QSUB;
-constexpr int OFF_RECV = OFF_P + P_BUF;          // chunk-merge buffer when at most 64 rows are in use
-constexpr int RECV_BYTES = 8 * 64 * (DH / 8 + 4) * 4;
-constexpr int SMEM_BYTES = OFF_RECV + RECV_BYTES;    // 200 KB
+constexpr int SMEM_BYTES = OFF_P + 2 * P_BUF;    // 224 KB
 constexpr int THREADS = 192;
 constexpr int E_TIMEOUT = 6;
-constexpr int TMEM_COLS = 256;               // S: 2 x 64 columns, O_t: 128 columns
+constexpr int TMEM_COLS = 256;               // S: 2 x 64 columns, O: 128 columns
 constexpr int COL_S = 0, COL_O = 128;
-static_assert(8 * 128 * (DH / 8 + 4) * 4 <= NKV * KV_STAGE + P_BUF && 128 * (DH + 4) * 4 <= NKV * KV_STAGE + P_BUF,
-              "with more than 64 rows the chunk-merge buffer fits in the K/V ring plus P");
-static_assert(64 * (DH + 4) * 4 <= RECV_BYTES && 2 * 64 * (DH / 2 + 4) * 4 <= RECV_BYTES && 4 * 64 * (DH / 4 + 4) * 4 <= RECV_BYTES,
-              "with at most 64 rows the chunk-merge buffer has room of its own");
+constexpr float RESCALE_STEP = 8.f;          // O is rescaled only when a row's maximum grows by more than 2^8
+// the chunk-merge buffer reuses the K/V ring once every CTA of the cluster is done with its tiles
+static_assert(8 * 128 * (DH / 8 + 4) * 4 <= NKV * KV_STAGE && 128 * (DH + 4) * 4 <= NKV * KV_STAGE,
+              "the chunk-merge buffer fits in the K/V ring");
 
 __device__ __forceinline__ void split_pack(float x, float y, uint32_t &hi, uint32_t &lo) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
@@ -116,6 +118,7 @@ struct AttnParams {
   RowPlan plan;
   bf16 *out, *out_lo;      // [R][n_heads * 128]
   int rows_per_seq, n_heads, S_max, chunks;
+  int longest_first;       // 1: grid slot y / n_heads takes the sequence with that rank in descending cache length
   int *status;
 };
 
@@ -131,7 +134,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   constexpr int NC = DUP ? 32 : 64;      // score columns (keys of a tile) per thread
   constexpr int ND = DUP ? 64 : 128;     // output dims per thread
   extern __shared__ unsigned char smem_raw[];
-  __shared__ uint64_t q_full, kv_full[NKV], kv_empty[NKV], s_full[2], p_full, o_full, x_bar[2], drain_bar;
+  __shared__ uint64_t q_full, kv_full[NKV], kv_empty[NKV], s_full[2], p_full[2], pv_done[2], x_bar[2], drain_bar;
   __shared__ float xch[2][128];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int s_error;
@@ -141,7 +144,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   unsigned char *sm = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
   const uint32_t sb = smem_u32(sm);
   const int c = blockIdx.x;
-  const int b = blockIdx.y / P.n_heads, h = blockIdx.y % P.n_heads;
+  int b = blockIdx.y / P.n_heads;
+  const int h = blockIdx.y % P.n_heads;
   const int H = P.n_heads * DH;
   const int n_q = (P.rows_per_seq + 31) >> 5;             // 32-row groups in use
   const int n_arrive = DUP ? 2 * n_q : n_q;               // row warps in use
@@ -150,11 +154,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   if (threadIdx.x == 0) {
     mbar_init(&q_full, 1);
     for (int s = 0; s < NKV; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
-    mbar_init(&p_full, (uint32_t)n_arrive);
-    mbar_init(&o_full, 1);
     mbar_init(&drain_bar, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s_full[i], 1);
+      mbar_init(&p_full[i], (uint32_t)n_arrive);
+      mbar_init(&pv_done[i], 1);
       mbar_init(&x_bar[i], 2);
     }
     s_error = 0;
@@ -176,6 +180,20 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   const uint32_t tmem = tmem_base_slot;
 
   pdl_wait();                      // Q, the tree rows of K/V and the row plan come from earlier kernels
+  if (P.longest_first) {
+    // More CTAs than SMs: the CTAs beyond the first round start when the first ones finish, so the
+    // sequences are taken longest first and the late CTAs belong to the shortest one.  Lane l holds
+    // sequence l's length; its rank is the number of sequences that are longer (ties: lower index).
+    const int nb = (int)gridDim.y / P.n_heads;              // <= 32 here
+    const int len_l = lane < nb ? P.plan.kv_len[lane] : -1;
+    int rank = 0;
+    for (int j = 0; j < nb; ++j) {
+      const int len_j = __shfl_sync(0xffffffffu, len_l, j);
+      rank += (len_j > len_l || (len_j == len_l && j < lane)) ? 1 : 0;
+    }
+    const unsigned hit = __ballot_sync(0xffffffffu, lane < nb && rank == b);
+    b = hit ? __ffs(hit) - 1 : b;
+  }
   if (threadIdx.x == 128) {        // warp 4 lane 0: the queries do not depend on the plan
     mbar_expect_tx(&q_full, (uint32_t)(4 * QSUB));
 #pragma unroll
@@ -265,11 +283,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       if (ok && T > 0) ok = issue_s(0);
       for (int t = 0; t < T && ok; ++t) {
         if (t + 1 < T) { ok = issue_s(t + 1); if (!ok) break; }
-        ok = mbar_wait(&p_full, (uint32_t)t & 1u);
+        ok = mbar_wait(&p_full[t & 1], (uint32_t)(t >> 1) & 1u);
         if (!ok) break;
         tc_fence_after();
         const uint32_t vb = sb + OFF_KV + (t % NKV) * KV_STAGE + 2 * SUB;
-        const uint32_t pb = sb + OFF_P;
+        const uint32_t pb = sb + OFF_P + (t & 1) * P_BUF;
         const uint32_t d = tmem + (uint32_t)COL_O;
 #pragma unroll
         for (int part = 0; part < 2; ++part) {            // P value, then P residual
@@ -277,49 +295,31 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
 #pragma unroll
           for (int k = 0; k < 4; ++k) {                    // 16 keys per MMA
             const uint64_t db = smem_desc_mn_sw128(vb + k * 2048, SUB, 1024);
-            umma_bf16(d, da + (uint64_t)(2 * k), db, idesc_o, (part | k) ? 1u : 0u);
+            umma_bf16(d, da + (uint64_t)(2 * k), db, idesc_o, (t | part | k) ? 1u : 0u);   // O accumulates over the tiles
           }
         }
         umma_commit(&kv_empty[t % NKV]);
-        umma_commit(&o_full);
+        umma_commit(&pv_done[t & 1]);
       }
       if (!ok) atomicExch(&s_error, 1);
     }
   } else if (row_warp) {
     // ------------------------------------------------------------------ softmax rows
+    // O accumulates in tensor memory over all tiles of the chunk.  A row's exponentials are taken
+    // relative to a reference maximum m_run that is raised only when a tile's maximum exceeds it
+    // by more than RESCALE_STEP (then the row's O and l are multiplied by 2^(old - new) in place);
+    // in between the probabilities may exceed 1 (by at most 2^RESCALE_STEP), which costs nothing in
+    // fp32 / bf16-pair arithmetic, and the rows never wait for P V except to reuse a P buffer.
     const int slot = P.plan.slot[r_glob];
     const bool ok_row = row_in && slot >= 0;
     const uint64_t mk0 = ok_row ? P.plan.mask[(size_t)r_glob * 2] : 0ull;
     const uint64_t mk1 = ok_row ? P.plan.mask[(size_t)r_glob * 2 + 1] : 0ull;
-#pragma unroll
-    for (int d = 0; d < ND; ++d) acc[d] = 0.f;
     const float sc = 0.08838834764831845f * 1.4426950408889634f;    // 1/sqrt(128) * log2(e)
     const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;          // this warp's 32 TMEM lanes
     const uint32_t prow = (uint32_t)(row * 128);
     const uint32_t psw = (uint32_t)(row & 7);
+    const uint32_t o_base = tmem + lane_sel + (uint32_t)(COL_O + ND * half);
     bool ok = true;
-    float m_prev = -INFINITY, l_prev = 0.f;
-
-    auto merge_o = [&](int u, float m_u, float l_u) -> bool {
-      if (!__all_sync(0xffffffffu, mbar_wait(&o_full, (uint32_t)u & 1u))) return false;
-      tc_fence_after();
-      const float m_new = fmaxf(m_run, m_u);
-      const float mu = m_new == -INFINITY ? 0.f : m_new;
-      const float a = exp2f(m_run - mu), bw = exp2f(m_u - mu);      // exp2(-inf) = 0
-      l_run = l_run * a + l_u * bw;
-      m_run = m_new;
-      const uint32_t base = tmem + lane_sel + (uint32_t)(COL_O + ND * half);
-#pragma unroll
-      for (int c0 = 0; c0 < ND; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld16(base + (uint32_t)c0, v);
-        tmem_ld16(base + (uint32_t)(c0 + 16), v + 16);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-        for (int j = 0; j < 32; ++j) acc[c0 + j] = acc[c0 + j] * a + __uint_as_float(v[j]) * bw;
-      }
-      return true;
-    };
 
     for (int t = 0; t < T; ++t) {
       ok = __all_sync(0xffffffffu, mbar_wait(&s_full[t & 1], (uint32_t)(t >> 1) & 1u));   // warp-uniform
@@ -356,6 +356,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       }
       if (DUP) {
         // the row's maximum over the whole tile: exchange with the thread that holds the other 32 keys
+        // (both threads of a row then keep the same reference maximum)
         xch[t & 1][threadIdx.x] = m_t;
         __syncwarp();
         if (lane == 0) mbar_arrive(&x_bar[rq]);
@@ -363,14 +364,41 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         if (!ok) break;
         m_t = fmaxf(m_t, xch[t & 1][threadIdx.x ^ 64]);
       }
-      // fold the previous tile's P V in first: that also tells that P and O_t may be overwritten
-      if (t >= 1) {
-        ok = merge_o(t - 1, m_prev, l_prev);
+      // raise the reference maximum?  (the first visible key sets it; O holds nothing of this row yet then)
+      float factor = 1.f;
+      if (m_t > m_run + RESCALE_STEP || (m_run == -INFINITY && m_t > -INFINITY)) {
+        factor = m_run == -INFINITY ? 0.f : exp2f(m_run - m_t);
+        m_run = m_t;
+      }
+      const bool rescale = t > 0 && __any_sync(0xffffffffu, factor != 1.f);
+      if (rescale) {
+        // every P V issued so far must have landed before O is touched; none can be issued before
+        // this warp has handed in its P of tile t
+        ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(t - 1) & 1], (uint32_t)((t - 1) >> 1) & 1u));
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int c0 = 0; c0 < ND; c0 += 16) {
+          uint32_t o[16];
+          tmem_ld16(o_base + (uint32_t)c0, o);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
+          tmem_st16(o_base + (uint32_t)c0, o);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        l_run *= factor;
+      } else if (t == 0) {
+        l_run = 0.f;
+      }
+      // the P buffer of tile t was last read by the P V of tile t - 2
+      if (t >= 2) {
+        ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[t & 1], (uint32_t)((t - 2) >> 1) & 1u));
         if (!ok) break;
       }
-      const float mu = m_t == -INFINITY ? 0.f : m_t;
+      const float mu = m_run == -INFINITY ? 0.f : m_run;
       float l_t = 0.f;
-      const uint32_t pb = sb + OFF_P + prow;
+      const uint32_t pb = sb + OFF_P + (uint32_t)((t & 1) * P_BUF) + prow;
 #pragma unroll
       for (int ch = 0; ch < NC / 8; ++ch) {
         uint32_t hi[4], lo[4];
@@ -389,14 +417,30 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
           st_shared_v4(pb + QSUB + 64 * 128 + off, lo[0], lo[1], lo[2], lo[3]);
         }
       }
+      l_run += l_t;
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full);
-      m_prev = m_t;
-      l_prev = l_t;
+      if (lane == 0) mbar_arrive(&p_full[t & 1]);
     }
-    if (ok && T > 0) ok = merge_o(T - 1, m_prev, l_prev);
+    // the chunk's unnormalised O (relative to m_run) out of tensor memory
+#pragma unroll
+    for (int d = 0; d < ND; ++d) acc[d] = 0.f;
+    if (ok && T > 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(T - 1) & 1], (uint32_t)((T - 1) >> 1) & 1u));
+      if (ok) {
+        tc_fence_after();
+#pragma unroll
+        for (int c0 = 0; c0 < ND; c0 += 32) {
+          uint32_t o[32];
+          tmem_ld16(o_base + (uint32_t)c0, o);
+          tmem_ld16(o_base + (uint32_t)(c0 + 16), o + 16);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < 32; ++j) acc[c0 + j] = __uint_as_float(o[j]);
+        }
+      }
+    }
     if (!ok) atomicExch(&s_error, 1);
   }
 
@@ -408,8 +452,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   const int wc = DH / P.chunks;
   const int rs = wc + 4;                 // floats per received row: wc dims, m, l (first keys), l (other keys), pad
   constexpr int RR = DUP ? 64 : 128;     // rows per source chunk in the receive buffer
-  float *recv = reinterpret_cast<float *>(sm + (DUP ? OFF_RECV : OFF_KV));
-  if (!DUP && P.chunks > 1) cluster_sync_all();  // every CTA of the cluster is done with its K/V ring
+  float *recv = reinterpret_cast<float *>(sm + OFF_KV);
+  if (P.chunks > 1) cluster_sync_all();  // the receive buffer reuses the K/V ring: every CTA of the cluster is done with its tiles
   if (row_in) {
     const uint32_t mine = smem_u32(recv + ((size_t)c * RR + row) * rs);
 #pragma unroll
@@ -480,30 +524,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
 }
 
 int g_attn_tc_min_rows = 16;   // fewer query rows per sequence than this: the mma.sync kernel
+int g_attn_tc_chunks = 0;      // > 0: this many key chunks whatever the shape (A/B runs)
 
 }  // namespace
 
 void attn_tc_set_min_rows(int rows) { g_attn_tc_min_rows = rows; }
+void attn_tc_set_chunks(int chunks) { g_attn_tc_chunks = chunks; }
 
-// Key chunks (= cluster size) per (sequence, head): 1, 2, 4 or 8, each chunk with at least 128 keys of
-// capacity.  One CTA per SM is resident, so `chunks * B * n_heads` CTAs run in rounds over the SMs; a
-// CTA costs a fixed part (set-up, the queries, the merge) plus its share of the key tiles.  The
-// estimate below, in microseconds from this kernel's measured tile and launch times, picks the
-// count with the shortest total (few sequences and heads: as many chunks as fill the SMs once;
-// more CTAs than SMs: shorter CTAs so that the last, partly filled round costs less).
+// Key chunks (= cluster size) per (sequence, head): the largest of 1, 2, 4, 8 that keeps the CTA
+// count within the SMs (one CTA per SM is resident; measured: a second, partly filled round and the
+// co-scheduling of clusters cost more than shorter CTAs gain), each chunk with at least 128 keys of
+// capacity.
 int attn_tc_chunks(int B, int n_heads, int S_max, int num_sms) {
-  const double fixed_us = 5.0, tile_us = 1.4;
-  const double tiles = (double)((S_max + TK - 1) / TK);
-  int best = 1;
-  double best_t = 0.0;
-  for (int c = 1; c <= 8; c *= 2) {
-    if (c > 1 && c * 128 > S_max) break;
-    const long long ctas = (long long)c * B * n_heads;
-    const double rounds = (double)((ctas + num_sms - 1) / num_sms);
-    const double t = rounds * (fixed_us + tile_us * tiles / c);
-    if (c == 1 || t < best_t - 1e-9) { best = c; best_t = t; }
+  int c = 1;
+  if (g_attn_tc_chunks > 0) {
+    while (2 * c <= g_attn_tc_chunks && 2 * c <= 8 && 2 * c * 128 <= S_max) c *= 2;
+    return c;
   }
-  return best;
+  while (c < 8 && 2 * c * B * n_heads <= num_sms && 2 * c * 128 <= S_max) c *= 2;
+  return c;
 }
 
 bool attn_tc_supported(int rows_per_seq, int head_dim, int S_max) {
@@ -528,7 +567,8 @@ cudaError_t tree_attention_tc(Launch L, Operand q_pair, int q_rows_alloc, const 
   if (!tc_get_map(q_pair.hi, q_rows_alloc, H, 64, &tmQh) || !tc_get_map(q_pair.lo, q_rows_alloc, H, 64, &tmQl) ||
       !tc_get_map(k_cache, (int)rows, DH, TK, &tmK) || !tc_get_map(v_cache, (int)rows, DH, TK, &tmV))
     return cudaErrorInvalidValue;
-  AttnParams P{plan, (bf16 *)out.hi, (bf16 *)out.lo, rows_per_seq, n_heads, S_max, chunks, status};
+  const int longest_first = (B > 1 && B <= 32 && (long long)chunks * B * n_heads > tc_num_sms()) ? 1 : 0;
+  AttnParams P{plan, (bf16 *)out.hi, (bf16 *)out.lo, rows_per_seq, n_heads, S_max, chunks, longest_first, status};
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(chunks, n_heads * B);
   cfg.blockDim = dim3(THREADS);

@@ -438,8 +438,10 @@ int tc_init_driver(char *err, size_t errlen) {
 }
 
 void attn_tc_set_min_rows(int rows);
+void attn_tc_set_chunks(int chunks);
 void tc_set_tuning(int key, int value) {
   if (key == 9) attn_tc_set_min_rows(value);
+  if (key == 12) attn_tc_set_chunks(value);
   if (key == 1) g_tune_stages = value;
   if (key == 10) g_tune_no_wave_split = value;
   if (key == 11) g_tune_no_wide = value;

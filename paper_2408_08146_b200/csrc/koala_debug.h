@@ -22,7 +22,8 @@ extern "C" {
  * stages request their weight tile before that wait (< 0 = all, the default); key 9 = fewest query
  * rows per sequence for which the tcgen05 attention kernel is used (default 16); key 10 = 1 keeps
  * the one-wave split-K factor when a launch has several token tiles (more than 128 rows);
- * key 11 = 1 keeps 128 weight rows per CTA also for the widest token tiles (MMA N = 256). */
+ * key 11 = 1 keeps 128 weight rows per CTA also for the widest token tiles (MMA N = 256);
+ * key 12 = key chunks per (sequence, head) of the tcgen05 attention kernel (0 = chosen from the shape). */
 void koala_set_tuning(int key, int value);
 
 /* Kernels launched by the library in this process so far (all contexts). */

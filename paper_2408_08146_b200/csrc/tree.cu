@@ -200,7 +200,8 @@ __global__ void plan_draft_p_kernel(TreeBufs t, PlanBufs p, const int32_t *seq_l
 
 // ------------------------------------------------------------------------------- dynamic expansion
 // Shared scratch: scores and flags of the candidates being ranked.
-__global__ void expand_dynamic_kernel(TreeBufs t, int k, int pool, int pass, int D, int N) {
+__global__ void __launch_bounds__(1024)
+expand_dynamic_kernel(TreeBufs t, int k, int pool, int pass, int D, int N) {
   extern __shared__ unsigned char smem_raw[];
   float *s_score = reinterpret_cast<float *>(smem_raw);            // [pool]
   int *s_node = reinterpret_cast<int *>(s_score + pool);           // [pool] node index or -1
@@ -269,9 +270,16 @@ __global__ void expand_dynamic_kernel(TreeBufs t, int k, int pool, int pass, int
   }
   if (pass != D - 1) return;
   // ---- final selection: the N-1 best candidates of the whole pool, numbered by
-  //      (level, parent's node number, rank)
+  //      (level, parent's node number, rank).  Scores, parents and the per-level ordering keys are
+  //      staged in shared memory once; every candidate has a thread of its own (the launcher gives
+  //      this pass enough threads), so each ranking loop is one pass over shared memory.
+  int *s_par = reinterpret_cast<int *>(s_mask + 2 * k);            // [pool] parent candidate id
+  int *s_key = s_par + pool;                                       // [pool] parent's node number * 32 + rank, -1 = dropped
   __syncthreads();
-  for (int c = tid; c < pool; c += nt) s_score[c] = t.cand_score[pb + c];
+  for (int c = tid; c < pool; c += nt) {
+    s_score[c] = t.cand_score[pb + c];
+    s_par[c] = t.cand_parent[pb + c];
+  }
   __syncthreads();
   for (int c = tid; c < pool; c += nt) {
     const float sc = s_score[c];
@@ -296,34 +304,26 @@ __global__ void expand_dynamic_kernel(TreeBufs t, int k, int pool, int pass, int
     const int lo = lvl == 1 ? 0 : k + (lvl - 2) * kk;
     const int hi = lvl == 1 ? k : k + (lvl - 1) * kk;
     const int base_node = s_base;
-    int my_node[8];          // a thread owns at most ceil(kk / nt) candidates of a level
-    int cnt = 0;
-    for (int c = lo + tid; c < hi; c += nt, ++cnt) {
-      my_node[cnt & 7] = -1;
-      if (s_node[c] != -2) continue;
-      const int par = t.cand_parent[pb + c];
-      const int pn = par < 0 ? 0 : s_node[par];
-      const int rk = t.cand_rank[pb + c];
+    // ordering key of every kept candidate of the level (the parents already have their numbers)
+    for (int c = lo + tid; c < hi; c += nt) {
+      const int par = s_par[c];
+      const int rk = lvl == 1 ? c : (c - lo) % k;
+      s_key[c] = s_node[c] == -2 ? (par < 0 ? 0 : s_node[par]) * 32 + rk : -1;
+    }
+    __syncthreads();
+    int kept_here = 0;
+    for (int c = lo + tid; c < hi; c += nt) {
+      const int key = s_key[c];
+      if (key < 0) continue;
       int before = 0;
       for (int f = lo; f < hi; ++f) {
-        if (f == c || s_node[f] == -1) continue;
-        const int fpar = t.cand_parent[pb + f];
-        const int fpn = fpar < 0 ? 0 : s_node[fpar];
-        const int frk = t.cand_rank[pb + f];
-        before += (fpn < pn || (fpn == pn && frk < rk)) ? 1 : 0;
+        const int kf = s_key[f];
+        before += (kf >= 0 && kf < key) ? 1 : 0;
       }
-      my_node[cnt & 7] = base_node + before;
-    }
-    __syncthreads();     // all reads of this level's s_node (-2 flags) are done
-    int kept_here = 0;
-    cnt = 0;
-    for (int c = lo + tid; c < hi; c += nt, ++cnt) {
-      const int node = my_node[cnt & 7];
-      if (node < 0) continue;
-      s_node[c] = node;
-      const int par = t.cand_parent[pb + c];
+      const int node = base_node + before;
+      s_node[c] = node;                     // read by the next level only (after the barrier below)
       t.tree_tok[b * N + node] = t.cand_tok[pb + c];
-      t.tree_parent[b * N + node] = par < 0 ? 0 : s_node[par];
+      t.tree_parent[b * N + node] = key >> 5;
       t.tree_level[b * N + node] = lvl;
       t.tree_score[b * N + node] = s_score[c];
       ++kept_here;
@@ -505,8 +505,12 @@ cudaError_t plan_medusa(Launch L, TreeBufs t, PlanBufs p, int B, int N, int head
                   B, N, heads);
 }
 cudaError_t expand_dynamic(Launch L, TreeBufs t, int B, int k, int pool, int pass, int D, int N) {
-  const size_t smem = (size_t)pool * 8 + (size_t)((k + 1) & ~1) * 4 + (size_t)k * 16 + 16;
-  return launch_k(expand_dynamic_kernel, dim3(B), dim3(256), smem, L.st, L.pdl, t, k, pool, pass, D, N);
+  const size_t smem = (size_t)pool * 16 + (size_t)((k + 1) & ~1) * 4 + (size_t)k * 16 + 16;
+  // the last pass ranks the whole pool: a thread per candidate
+  int threads = 256;
+  if (pass == D - 1)
+    while (threads < pool && threads < 1024) threads *= 2;
+  return launch_k(expand_dynamic_kernel, dim3(B), dim3(threads), smem, L.st, L.pdl, t, k, pool, pass, D, N);
 }
 cudaError_t expand_static(Launch L, TreeBufs t, const int32_t *s_parent, const int32_t *s_level,
                           const int32_t *s_rank, int B, int N, int k) {

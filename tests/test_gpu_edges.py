@@ -141,13 +141,28 @@ def test_unwritten_cache_slots_may_hold_nan(N, B, n_heads, context, S_max):
     _attention_case(N, B, n_heads, context, S_max, poison=True)
 
 
-def _attention_case(N, B, n_heads, context, S_max, poison=False):
+@pytest.mark.parametrize("N,B,n_heads,context,S_max", [
+    (60, 1, 32, 1000, 2048),     # duplicated rows, 4 key chunks of several tiles each
+    (128, 1, 32, 1500, 4096),    # every row warp owns its rows
+])
+def test_scores_that_grow_along_the_context(N, B, n_heads, context, S_max):
+    """Keys whose magnitude grows eightfold from the first to the last cached position: the row
+    maxima rise by far more than 2^8 from tile to tile, so the running output, which the tcgen05
+    kernel keeps in tensor memory relative to a lazily raised reference maximum, is rescaled in place
+    several times."""
+    _attention_case(N, B, n_heads, context, S_max, growing=True)
+
+
+def _attention_case(N, B, n_heads, context, S_max, poison=False, growing=False):
     H = n_heads * 128
     cfg = reduced(T7_EAGLE, 1, K=1, N=N, B=B, H=H, n_heads=n_heads, F=2 * H, V=2048, D=min(5, N - 1),
                   S_max=S_max, prompt_len=context)
     eng, orc, _ = make_pair(cfg, oracle_dtype=np.float32, cache_host=False)
     eng.target_k.copy_(random_kv(cfg, "target_k", cfg.L, DEV))
     eng.target_v.copy_(random_kv(cfg, "target_v", cfg.L, DEV))
+    if growing:
+        ramp = 1.0 + 7.0 * torch.arange(S_max, device=DEV, dtype=torch.float32) / context
+        eng.target_k.copy_((eng.target_k.float() * ramp.view(1, 1, 1, S_max, 1)).to(eng.target_k.dtype))
     lens = [context - 13 * b for b in range(B)]
     for b in range(B):
         orc.target_k[0][b][...] = kv_to_oracle(eng.target_k, 0, b, np.float32)
