@@ -39,7 +39,7 @@ __device__ __forceinline__ float warp_max(float v) {
 
 // A matrix given as the sum of partial matrices `stride` floats apart (split-K results).
 // Classic split-K: every column has `n` partials.  Stream-K (sk_ctas > 0): column c belongs to
-// weight tile c / 128, whose K-blocks were dealt to the CTAs owning units
+// weight tile c / 128 (c / 256 with sk_wide), whose K-blocks were dealt to the CTAs owning units
 // [tile * sk_kb, (tile + 1) * sk_kb); it has one partial per such CTA, in slots 0, 1, ...
 struct SplitIn {
   const float *p;
@@ -47,9 +47,10 @@ struct SplitIn {
   size_t stride;
   int ld;
   unsigned sk_ctas, sk_units, sk_kb;
+  unsigned sk_wide;        // stream-K: 1 = the weight tiles are 256 columns wide instead of 128
   __device__ __forceinline__ int count(int c) const {
     if (sk_ctas == 0) return n;
-    const unsigned u0 = (unsigned)(c >> 7) * sk_kb;
+    const unsigned u0 = (unsigned)(c >> (7 + sk_wide)) * sk_kb;
     const unsigned first = ((u0 + 1u) * sk_ctas - 1u) / sk_units;
     const unsigned last = ((u0 + sk_kb) * sk_ctas - 1u) / sk_units;
     return (int)(last - first) + 1;

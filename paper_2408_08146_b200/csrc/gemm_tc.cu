@@ -66,6 +66,9 @@ struct TcParams {
   size_t split_stride;
   int stages;
   int wide;           // 1: 256 weight rows per CTA (two accumulators), N = 256, one CTA per SM
+  int accp;           // 1: the pair's residual rows are a second, accumulating MMA into the same columns
+                      //    (bn = tt: up to 256 tokens per tile) instead of extra columns (bn = 2 tt)
+  int pf_ahead;       // weight tiles requested into L2 this many units ahead of the ring (0 = none)
   int early_w;        // how many of the first stages' weight tiles are requested before the dependency wait
   int l2_ahead;       // weight tiles prefetched into L2 beyond the ring before the dependency wait
   int *status;
@@ -92,7 +95,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char *tiles = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
-  const int x_stage_bytes = P.bn * BK * 2;
+  const int x_stage_bytes = (P.accp ? 2 : 1) * P.bn * BK * 2;
   const int w_stage_bytes = P.wide ? 2 * W_STAGE_BYTES : W_STAGE_BYTES;
   const int stage_bytes = w_stage_bytes + x_stage_bytes;   // both multiples of 1024
   const int bm = P.wide ? 2 * BM : BM;                     // weight rows per tile
@@ -198,7 +201,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       bool ok = true;
       int s = pre % P.stages;
       uint32_t ph = (uint32_t)(pre / P.stages) & 1u;
+      // Optional (tuning key 14): the weight tiles of the units `pf_ahead` beyond the one being loaded are
+      // requested into L2.  With the two 96 KB stages of the 256-token mode this was measured slower
+      // than no lookahead (13B shapes: 18.2 against 17.7 ms per verification), so it is off.
+      int pf_tile = tile, pf_kb = kb, pf_row0 = row0, pf_it = pre;
+      const CUtensorMap *pf_map = tmW;
+      auto pf_step = [&]() {
+        if (++pf_kb == KB) { pf_kb = 0; ++pf_tile; pf_map = tile_map(pf_tile, pf_row0); }
+        ++pf_it;
+      };
+      auto pf_request = [&]() {
+        asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+                     ::"l"(pf_map), "r"(pf_kb * BK), "r"(pf_row0) : "memory");
+        if (P.wide)
+          asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+                       ::"l"(pf_map), "r"(pf_kb * BK), "r"(pf_row0 + BM) : "memory");
+      };
+      if (P.pf_ahead > 0) {
+        for (int q = 0; q < P.pf_ahead && pf_it < n_units; ++q) { pf_request(); pf_step(); }
+      }
       for (int it = pre; it < n_units; ++it) {
+        if (P.pf_ahead > 0 && pf_it < n_units) { pf_request(); pf_step(); }
         ok = mbar_wait(&empty_bar[s], ph ^ 1u);
         if (!ok) break;
         mbar_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
@@ -240,15 +263,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         const uint64_t da = smem_desc_sw128(wa);
         const uint64_t da2 = smem_desc_sw128(wa + W_STAGE_BYTES);      // wide: the second 128 weight rows
         const uint64_t db = smem_desc_sw128(wa + (uint32_t)w_stage_bytes);
+        const uint64_t db2 = smem_desc_sw128(wa + (uint32_t)(w_stage_bytes + P.tt * BK * 2));   // accp: the residual rows
         const uint32_t dacc = tmem_acc + (uint32_t)(buf * P.tmem_cols);
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; ++k) {
           // advance 32 bytes (16 bf16) inside the swizzled row: +2 in the 16-byte address field
-          umma_bf16(dacc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
-                    (!seg_start || k > 0) ? 1u : 0u);
-          if (P.wide)
-            umma_bf16(dacc + (uint32_t)P.tmem_cols, da2 + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
-                      (!seg_start || k > 0) ? 1u : 0u);
+          const uint32_t acc = (!seg_start || k > 0) ? 1u : 0u;
+          umma_bf16(dacc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, acc);
+          if (P.accp) umma_bf16(dacc, da + (uint64_t)(2 * k), db2 + (uint64_t)(2 * k), idesc, 1u);
+          if (P.wide) {
+            umma_bf16(dacc + (uint32_t)P.tmem_cols, da2 + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, acc);
+            if (P.accp) umma_bf16(dacc + (uint32_t)P.tmem_cols, da2 + (uint64_t)(2 * k), db2 + (uint64_t)(2 * k), idesc, 1u);
+          }
         }
         umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
         const bool seg_end = (kb == KB - 1) || it == n_units - 1;
@@ -293,14 +319,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       for (int c0 = 0; c0 < P.tt; c0 += 16) {
         uint32_t v[16], w[16];
         tmem_ld16(lane_base + (uint32_t)c0, v);
-        if (P.pair) tmem_ld16(lane_base + (uint32_t)(P.tt + c0), w);
+        if (P.pair && !P.accp) tmem_ld16(lane_base + (uint32_t)(P.tt + c0), w);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (feat < n_rows) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int t = tok0 + c0 + j;
             float r = __uint_as_float(v[j]);
-            if (P.pair) r += __uint_as_float(w[j]);
+            if (P.pair && !P.accp) r += __uint_as_float(w[j]);
             if (t < P.R) Yp[(size_t)t * P.ldy] = r;
           }
         }
@@ -368,6 +394,8 @@ int g_tune_l2_ahead = -1;   // < 0 = default
 int g_tune_late_w = 0;      // 1 = weights wait for the dependency too
 int g_tune_early_stages = -1; // < 0 = all stages
 int g_tune_no_wave_split = 0; // 1 = several token tiles keep the one-wave rule's split factor
+int g_tune_no_accp = 0;      // 1 = pairs of more than 128 tokens as two 128-token tiles with extra columns
+int g_tune_pf = 0;           // > 0: weight tiles requested into L2 ahead of the ring in that mode
 int g_tune_no_wide = 0;      // 1 = 128 weight rows per CTA also for wide token tiles
 int g_tune_traffic_div = 8; // split <= K_in / (div * tokens)
 
@@ -445,6 +473,8 @@ void tc_set_tuning(int key, int value) {
   if (key == 1) g_tune_stages = value;
   if (key == 10) g_tune_no_wave_split = value;
   if (key == 11) g_tune_no_wide = value;
+  if (key == 13) g_tune_no_accp = value;
+  if (key == 14) g_tune_pf = value;
   if (key == 2) g_tune_max_split = value;
   if (key == 3) g_tune_no_streamk = value;
   if (key == 5) g_tune_l2_ahead = value;
@@ -538,16 +568,22 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   TcParams P;
   memset(&P, 0, sizeof(P));
   const int pair = X.lo != nullptr ? 1 : 0;
-  const int tt_max = pair ? 128 : 256;
+  // A pair of more than 128 tokens keeps all of a tile's tokens in one accumulator (two accumulating
+  // MMAs per K step, value rows then residual rows) so that a tile holds up to 256 tokens and the
+  // weights are passed over once; up to 128 tokens the residual rows are extra accumulator columns.
+  const int accp = (pair && R > 128 && !g_tune_no_accp) ? 1 : 0;
+  const int tt_max = (pair && !accp) ? 128 : 256;
   int tt = ((R + 15) / 16) * 16;
   if (tt > tt_max) tt = tt_max;
   if (tt > x_rows_alloc) return cudaErrorInvalidValue;
-  const int bn = pair ? 2 * tt : tt;
+  const int bn = (pair && !accp) ? 2 * tt : tt;
+  const int x_bytes = (accp ? 2 : 1) * bn * BK * 2;      // activation bytes of a stage
   const int ztiles = (R + tt - 1) / tt;
   // the last token tile may reach past R: those rows must exist (they are read, results dropped)
   if (ztiles * tt > x_rows_alloc) return cudaErrorInvalidValue;
   P.tt = tt;
   P.pair = pair;
+  P.accp = accp;
   P.ztiles = ztiles;
   int cols = 32;
   while (cols < bn) cols <<= 1;
@@ -557,7 +593,7 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   P.bn = bn;
   P.tmem_cols = cols;
   // wide mode: N = 256, every matrix a whole number of 256-row tiles, room for three 64 KB stages
-  bool wide = !g_tune_no_wide && bn == 256 && g_smem_optin - 2048 >= 3 * (2 * W_STAGE_BYTES + bn * BK * 2);
+  bool wide = !g_tune_no_wide && bn == 256 && g_smem_optin - 2048 >= (accp ? 2 : 3) * (2 * W_STAGE_BYTES + x_bytes);
   for (int i = 0; i < m.n && wide; ++i) wide = (m.n_out[i] % (2 * BM)) == 0;
   const int bmw = wide ? 2 * BM : BM;
   P.wide = wide ? 1 : 0;
@@ -573,19 +609,40 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   P.kblocks = K_in / BK;
   // stream-K (split == 0): needs a single token tile and 128-row-aligned matrices, so that a
   // column's tile (and with it the number of partial sums to add) follows from the column index
-  bool sk = split == 0 && ztiles == 1 && max_slots >= 2 && out != nullptr && !g_tune_no_streamk && !wide;
-  for (int i = 0; i < m.n && sk; ++i) sk = (m.n_out[i] % BM) == 0;
+  bool sk = split == 0 && ztiles == 1 && max_slots >= 2 && out != nullptr && !g_tune_no_streamk;
+  for (int i = 0; i < m.n && sk; ++i) sk = (m.n_out[i] % bmw) == 0;
   // stream-K pays off where the per-tile decomposition cannot be split further and leaves the SMs
   // unevenly loaded (more tiles than SMs, not a whole number of two-per-SM waves); elsewhere
-  // classic split-K gives the same balance with fewer partial sums per tile
-  if (sk) {
+  // classic split-K gives the same balance with fewer partial sums per tile.  With 256-row tiles
+  // (one CTA per SM, tensor-bound) it is taken whenever the best split factor would leave more
+  // than a tenth of the SM-rounds empty.
+  int sk_ctas = 0, sk_slots = 1;
+  if (sk && wide) {
+    const int sp = wave_split(n_tiles, P.kblocks, R, 1, g_num_sms);
+    const int ctas = n_tiles * sp, rounds = (ctas + g_num_sms - 1) / g_num_sms;
+    sk = (double)ctas < 0.9 * (double)rounds * g_num_sms;
+    if (sk) {
+      // every CTA at least 8 K-blocks, at most max_slots contributors per tile
+      const long long units = (long long)n_tiles * P.kblocks;
+      long long g = g_num_sms;
+      if (g > units / 8) g = units / 8;
+      if (g < 1) g = 1;
+      auto slots_of = [&](long long gg) {
+        const long long per = units / gg;
+        return (int)((P.kblocks + per - 1) / per) + ((units % gg) || (P.kblocks % per) ? 1 : 0);
+      };
+      while (g > 1 && slots_of(g) > max_slots) --g;
+      sk_ctas = (int)g;
+      sk_slots = slots_of(g);
+      if (sk_ctas <= ctas) sk = false;          // the classic decomposition uses as many CTAs
+    }
+  } else if (sk) {
     const int classic = tc_default_split(n_tiles, P.kblocks, R);
     sk = classic == 1 && n_tiles > g_num_sms && (n_tiles % (2 * g_num_sms)) != 0;
-  }
-  int sk_ctas = 0, sk_slots = 1;
-  if (sk) {
-    sk_ctas = tc_streamk_ctas(n_tiles, P.kblocks, R, max_slots, &sk_slots);
-    if (sk_ctas <= n_tiles) sk = false;         // nothing to share: one CTA per tile is the same thing
+    if (sk) {
+      sk_ctas = tc_streamk_ctas(n_tiles, P.kblocks, R, max_slots, &sk_slots);
+      if (sk_ctas <= n_tiles) sk = false;         // nothing to share: one CTA per tile is the same thing
+    }
   }
   if (!sk) {
     sk_ctas = 0;
@@ -605,7 +662,7 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   P.split_stride = split_stride;
   P.status = status;
   P.nbuf = (sk && 2 * cols <= 256) ? 2 : 1;
-  const int stage_bytes = (wide ? 2 : 1) * W_STAGE_BYTES + bn * BK * 2;
+  const int stage_bytes = (wide ? 2 : 1) * W_STAGE_BYTES + x_bytes;
   int stages = (g_smem_optin - 2048) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages > 8) stages = 8;
@@ -617,6 +674,7 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   if (stages < 2) return cudaErrorInvalidValue;
   P.stages = stages;
   P.l2_ahead = g_tune_l2_ahead >= 0 ? g_tune_l2_ahead : L2_AHEAD;
+  P.pf_ahead = (accp && stages < 4 && g_tune_pf > 0) ? g_tune_pf : 0;   // measured: no lookahead is fastest (13B, 256 rows)
   P.early_w = g_tune_late_w ? 0 : (g_tune_early_stages >= 0 && g_tune_early_stages < stages ? g_tune_early_stages : stages);
   CUtensorMap mw[3], mx, mxlo;
   for (int i = 0; i < 3; ++i) {
@@ -629,7 +687,7 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   if (out) {
     *out = SplitIn{Y, sk ? sk_slots : split, split_stride, ldy, sk ? (unsigned)sk_ctas : 0u, P.sk_units,
-                   (unsigned)P.kblocks};
+                   (unsigned)P.kblocks, (sk && wide) ? 1u : 0u};
   }
   return launch_k(gemm_tc_kernel, grid, dim3(THREADS), smem, L.st, L.pdl, mw[0], mw[1], mw[2], mx, mxlo, P);
 }

@@ -992,7 +992,7 @@ void koala_destroy(koala_ctx *c) {
 
 int koala_gemm_x_rows(int M, int has_lo) {
   if (M < 1) return 0;
-  const int tt_max = has_lo ? 128 : 256;
+  const int tt_max = (has_lo && M <= 128) ? 128 : 256;    // as in the multiply: pairs of more than 128 tokens use 256-token tiles
   int tt = (M + 15) / 16 * 16;
   if (tt > tt_max) tt = tt_max;
   return (M + tt - 1) / tt * tt;

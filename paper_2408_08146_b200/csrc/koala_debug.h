@@ -23,7 +23,10 @@ extern "C" {
  * rows per sequence for which the tcgen05 attention kernel is used (default 16); key 10 = 1 keeps
  * the one-wave split-K factor when a launch has several token tiles (more than 128 rows);
  * key 11 = 1 keeps 128 weight rows per CTA also for the widest token tiles (MMA N = 256);
- * key 12 = key chunks per (sequence, head) of the tcgen05 attention kernel (0 = chosen from the shape). */
+ * key 12 = key chunks per (sequence, head) of the tcgen05 attention kernel (0 = chosen from the shape);
+ * key 13 = 1 runs pairs of more than 128 tokens as 128-token tiles with the residual rows as extra
+ * accumulator columns (the form used up to 128 tokens) instead of 256-token tiles with two accumulating
+ * MMAs; key 14 = weight tiles requested into L2 ahead of the ring in the 256-token form (default 0). */
 void koala_set_tuning(int key, int value);
 
 /* Kernels launched by the library in this process so far (all contexts). */
