@@ -103,7 +103,9 @@ def step_roofline(cfg, context: float, ms_per_step: float, peaks: dict) -> dict:
     t_tc = w["flops"] / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
     bound_ms = max(t_hbm, t_tc)
     return {"algorithmic_bytes_per_step": nbytes, "algorithmic_flops_per_step": w["flops"],
-            "ideal_ms_hbm": t_hbm, "ideal_ms_tensor": t_tc, "bound": "hbm" if t_hbm >= t_tc else "tensor",
+            "ideal_ms_hbm": t_hbm, "ideal_ms_tensor": t_tc,
+            # bf16 activations enter the MMAs as a value + residual pair: twice the algorithmic flops are issued
+            "ideal_ms_tensor_issued": 2.0 * t_tc if cfg.dtype == 1 else t_tc, "bound": "hbm" if t_hbm >= t_tc else "tensor",
             "achieved_GBps": nbytes / (ms_per_step * 1e-3) / 1e9, "achieved_TFLOPs": w["flops"] / (ms_per_step * 1e-3) / 1e12,
             "frac_of_peak": bound_ms / ms_per_step, "peak_source": f"of {peaks['source']}"}
 
