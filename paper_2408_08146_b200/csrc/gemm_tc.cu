@@ -14,11 +14,11 @@
 // token tile then holds the hi rows followed by the lo rows of the same tokens (MMA N doubles),
 // and the epilogue adds the two halves of the accumulator, so the product carries 16 significant
 // bits of the activations at no extra weight traffic.
-// Wide token tiles (MMA N = 256: more than 64 tokens as pairs): a pipeline stage would be 16 KB of
-// weights + 32 KB of activations, and the ring is bound by its capacity (bytes in flight /
-// latency), two thirds of it activations.  There a CTA takes 256 weight rows instead: two MMAs per
-// K step share the activation tile and fill two accumulators (all 512 tensor-memory columns), a
-// stage is 32 + 32 KB, one CTA per SM with three stages keeps 1.5 times the weight bytes in flight.
+// More than 128 tokens as a pair: value rows and residual rows are two accumulating MMAs into the same
+// accumulator columns, so a tile holds up to 256 tokens and the weights are passed over once.  With
+// 256 tokens a CTA takes 256 weight rows: four MMAs per K step share the activation tile and fill two
+// accumulators (all 512 tensor-memory columns); a stage is 32 KB of weights + 64 KB of activations,
+// two stages, one CTA per SM.
 // Split-K: grid.y CTAs share a weight tile and write separate partial outputs that the consumer
 // kernel sums in a fixed order (deterministic).
 // Every wait is bounded: on expiry the kernel records KOALA_E_TIMEOUT in *status, drains, frees
@@ -593,7 +593,9 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   P.bn = bn;
   P.tmem_cols = cols;
   // wide mode: N = 256, every matrix a whole number of 256-row tiles, room for three 64 KB stages
-  bool wide = !g_tune_no_wide && bn == 256 && g_smem_optin - 2048 >= (accp ? 2 : 3) * (2 * W_STAGE_BYTES + x_bytes);
+  // (At exactly 128 tokens, where the extra-column form also reaches N = 256, 128 weight rows per CTA with
+  // two CTAs per SM measured 6-7 % faster than 256 rows with one: 7B verify 5.7 against 6.1 ms.)
+  bool wide = !g_tune_no_wide && accp && bn == 256 && g_smem_optin - 2048 >= 2 * (2 * W_STAGE_BYTES + x_bytes);
   for (int i = 0; i < m.n && wide; ++i) wide = (m.n_out[i] % (2 * BM)) == 0;
   const int bmw = wide ? 2 * BM : BM;
   P.wide = wide ? 1 : 0;
