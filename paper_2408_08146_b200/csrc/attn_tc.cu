@@ -15,11 +15,7 @@
 // MMAs as bf16 pairs (value + rounding residual: two accumulating MMAs), so only the cached K and V
 // carry bf16 rounding.  Q (written as a pair by the rotary-embedding kernel) and the K/V tiles
 // arrive by TMA with the 128-byte swizzle, K/V in a three-stage ring.
-// Eight row warps in two groups: group 0 (warps 0..3) takes the even tiles of the chunk, group 1
-// (warps 4..7) the odd ones, each with an S buffer, a P buffer and an O accumulator of its own, so
-// that two tiles are in the rows' hands at any time (a tile costs the rows about 1.1 us of their own
-// instructions, the tensor pipe about half of that); the groups' results are merged through shared
-// memory at the end.  Warp 8 lane 0 issues the copies, warp 9 lane 0 the MMAs.
+// Warps 0..3 own the rows, warp 4 lane 0 issues the copies, warp 5 lane 0 the MMAs.
 // With several chunks the CTAs of one (head, sequence) form a thread-block cluster: every CTA
 // pushes, into each peer's shared memory, that peer's slice of the head dimension of its
 // unnormalised (O, m, l); after a cluster barrier every CTA merges its slice over the chunks in
@@ -51,11 +47,9 @@ constexpr int KV_STAGE = 4 * SUB;
 constexpr int OFF_P = OFF_KV + NKV * KV_STAGE;   // two buffers of P hi, P lo
 constexpr int P_BUF = 2 * QSUB;
 constexpr int SMEM_BYTES = OFF_P + 2 * P_BUF;    // 224 KB
-constexpr int ROW_WARPS = 8;                 // two groups of four row warps: group g takes the tiles t with t % 2 == g
-constexpr int TMA_WARP = ROW_WARPS, MMA_WARP = ROW_WARPS + 1;
-constexpr int THREADS = 32 * (ROW_WARPS + 2);
+constexpr int THREADS = 192;
 constexpr int E_TIMEOUT = 6;
-constexpr int TMEM_COLS = 512;               // S: 2 x 64 columns, O: 128 columns per group (128.., 256..)
+constexpr int TMEM_COLS = 256;               // S: 2 x 64 columns, O: 128 columns
 constexpr int COL_S = 0, COL_O = 128;
 constexpr float RESCALE_STEP = 8.f;          // O is rescaled only when a row's maximum grows by more than 2^8
 // the chunk-merge buffer reuses the K/V ring once every CTA of the cluster is done with its tiles
@@ -140,8 +134,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   constexpr int NC = DUP ? 32 : 64;      // score columns (keys of a tile) per thread
   constexpr int ND = DUP ? 64 : 128;     // output dims per thread
   extern __shared__ unsigned char smem_raw[];
-  __shared__ uint64_t q_full, kv_full[NKV], kv_empty[NKV], s_full[2], p_full[2], pv_done[2], x_bar[2][2], drain_bar;
-  __shared__ uint16_t xch[2][2][128];  // [group][tile parity within the group][thread of the group]: bf16 bits
+  __shared__ uint64_t q_full, kv_full[NKV], kv_empty[NKV], s_full[2], p_full[2], pv_done[2], x_bar[2], drain_bar;
+  __shared__ float xch[2][128];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int s_error;
 
@@ -165,8 +159,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       mbar_init(&s_full[i], 1);
       mbar_init(&p_full[i], (uint32_t)n_arrive);
       mbar_init(&pv_done[i], 1);
-      mbar_init(&x_bar[i][0], 2);
-      mbar_init(&x_bar[i][1], 2);
+      mbar_init(&x_bar[i], 2);
     }
     s_error = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -176,7 +169,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmK) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmV) : "memory");
   }
-  if (warp == MMA_WARP) {
+  if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -201,7 +194,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     const unsigned hit = __ballot_sync(0xffffffffu, lane < nb && rank == b);
     b = hit ? __ffs(hit) - 1 : b;
   }
-  if (threadIdx.x == 32 * TMA_WARP) {        // the queries do not depend on the plan
+  if (threadIdx.x == 128) {        // warp 4 lane 0: the queries do not depend on the plan
     mbar_expect_tx(&q_full, (uint32_t)(4 * QSUB));
 #pragma unroll
     for (int part = 0; part < 2; ++part)
@@ -220,19 +213,17 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   const int tile_hi = (int)(((long long)n_tiles * (c + 1)) / P.chunks);
   const int T = tile_hi - tile_lo;
 
-  // row ownership of the row warps: warps 0..3 are group 0 (even tiles), warps 4..7 group 1 (odd tiles)
-  const int grp = warp >> 2, wq = warp & 3;                 // wq also selects the warp's 32 tensor-memory lanes
-  const int gtid = threadIdx.x & 127;                       // thread index inside the group
-  const int rq = DUP ? (wq & 1) : wq;                       // 32-row group
-  const int half = DUP ? (wq >> 1) : 0;                     // which half of the keys / dims
+  // row ownership of warps 0..3
+  const int rq = DUP ? (warp & 1) : warp;                   // 32-row group
+  const int half = DUP ? (warp >> 1) : 0;                   // which half of the keys / dims
   const int row = rq * 32 + lane;
-  const bool row_warp = warp < ROW_WARPS && rq < n_q;
+  const bool row_warp = warp < 4 && rq < n_q;
   const bool row_in = row_warp && row < P.rows_per_seq;
   const int r_glob = b * P.rows_per_seq + (row_in ? row : 0);
   float acc[ND];
   float m_run = -INFINITY, l_run = 0.f;
 
-  if (warp == TMA_WARP) {
+  if (warp == 4) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       const int y0 = (b * P.n_heads + h) * P.S_max;
@@ -261,7 +252,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       }
       if (T == 0 || !ok) (void)mbar_wait(&q_full, 0);      // nobody else waits for Q then
     }
-  } else if (warp == MMA_WARP) {
+  } else if (warp == 5) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       // D fp32, A and B bf16; S: N = 64, both K-major; O_t: N = 128, B MN-major
@@ -297,14 +288,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         tc_fence_after();
         const uint32_t vb = sb + OFF_KV + (t % NKV) * KV_STAGE + 2 * SUB;
         const uint32_t pb = sb + OFF_P + (t & 1) * P_BUF;
-        const uint32_t d = tmem + (uint32_t)(COL_O + (t & 1) * DH);     // the O of the group that owns tile t
+        const uint32_t d = tmem + (uint32_t)COL_O;
 #pragma unroll
         for (int part = 0; part < 2; ++part) {            // P value, then P residual
           const uint64_t da = smem_desc_sw128(pb + part * QSUB);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {                    // 16 keys per MMA
             const uint64_t db = smem_desc_mn_sw128(vb + k * 2048, SUB, 1024);
-            umma_bf16(d, da + (uint64_t)(2 * k), db, idesc_o, ((t >> 1) | part | k) ? 1u : 0u);   // accumulates over the group's tiles
+            umma_bf16(d, da + (uint64_t)(2 * k), db, idesc_o, (t | part | k) ? 1u : 0u);   // O accumulates over the tiles
           }
         }
         umma_commit(&kv_empty[t % NKV]);
@@ -324,15 +315,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     const uint64_t mk0 = ok_row ? P.plan.mask[(size_t)r_glob * 2] : 0ull;
     const uint64_t mk1 = ok_row ? P.plan.mask[(size_t)r_glob * 2 + 1] : 0ull;
     const float sc = 0.08838834764831845f * 1.4426950408889634f;    // 1/sqrt(128) * log2(e)
-    const uint32_t lane_sel = (uint32_t)(wq * 32) << 16;            // this warp's 32 TMEM lanes
+    const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;          // this warp's 32 TMEM lanes
     const uint32_t prow = (uint32_t)(row * 128);
     const uint32_t psw = (uint32_t)(row & 7);
-    const uint32_t o_base = tmem + lane_sel + (uint32_t)(COL_O + grp * DH + ND * half);   // the group's own O
+    const uint32_t o_base = tmem + lane_sel + (uint32_t)(COL_O + ND * half);
     bool ok = true;
-    int t_last = -1;
 
-    for (int t = grp; t < T; t += 2) {          // the group's tiles; (t >> 1) counts them
-      t_last = t;
+    for (int t = 0; t < T; ++t) {
       ok = __all_sync(0xffffffffu, mbar_wait(&s_full[t & 1], (uint32_t)(t >> 1) & 1u));   // warp-uniform
       if (!ok) break;
       tc_fence_after();
@@ -368,17 +357,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       if (DUP) {
         // the row's maximum over the whole tile: exchange with the thread that holds the other 32 keys
         // (both threads of a row then keep the same reference maximum)
-        // Each thread rounds its maximum UP to a bf16 value and both take the larger of the two rounded
-        // values: identical in both threads, and never below the true maximum (any common reference
-        // serves; the probabilities stay <= 1 relative to it).
-        const uint32_t mb = __float_as_uint(m_t);
-        const uint32_t up = (mb & 0x80000000u) ? (mb & 0xffff0000u) : ((mb + 0xffffu) & 0xffff0000u);
-        xch[grp][(t >> 1) & 1][gtid] = (uint16_t)(up >> 16);
+        xch[t & 1][threadIdx.x] = m_t;
         __syncwarp();
-        if (lane == 0) mbar_arrive(&x_bar[grp][rq]);
-        ok = __all_sync(0xffffffffu, mbar_wait(&x_bar[grp][rq], (uint32_t)(t >> 1) & 1u));
+        if (lane == 0) mbar_arrive(&x_bar[rq]);
+        ok = __all_sync(0xffffffffu, mbar_wait(&x_bar[rq], (uint32_t)t & 1u));
         if (!ok) break;
-        m_t = fmaxf(__uint_as_float(up), __uint_as_float((uint32_t)xch[grp][(t >> 1) & 1][gtid ^ 64] << 16));
+        m_t = fmaxf(m_t, xch[t & 1][threadIdx.x ^ 64]);
       }
       // raise the reference maximum?  (the first visible key sets it; O holds nothing of this row yet then)
       float factor = 1.f;
@@ -386,14 +370,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         factor = m_run == -INFINITY ? 0.f : exp2f(m_run - m_t);
         m_run = m_t;
       }
-      // The group's previous tile is t - 2: its P V read the P buffer this tile is about to fill
-      // and wrote the O a rescale would touch; the P V of tile t cannot be issued before this warp
-      // has handed in its P.
-      if (t >= 2) {
-        ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[t & 1], (uint32_t)((t - 2) >> 1) & 1u));
+      const bool rescale = t > 0 && __any_sync(0xffffffffu, factor != 1.f);
+      if (rescale) {
+        // every P V issued so far must have landed before O is touched; none can be issued before
+        // this warp has handed in its P of tile t
+        ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(t - 1) & 1], (uint32_t)((t - 1) >> 1) & 1u));
         if (!ok) break;
-      }
-      if (t >= 2 && __any_sync(0xffffffffu, factor != 1.f)) {
         tc_fence_after();
 #pragma unroll
         for (int c0 = 0; c0 < ND; c0 += 16) {
@@ -406,6 +388,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         }
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         l_run *= factor;
+      } else if (t == 0) {
+        l_run = 0.f;
+      }
+      // the P buffer of tile t was last read by the P V of tile t - 2
+      if (t >= 2) {
+        ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[t & 1], (uint32_t)((t - 2) >> 1) & 1u));
+        if (!ok) break;
       }
       const float mu = m_run == -INFINITY ? 0.f : m_run;
       float l_t = 0.f;
@@ -437,8 +426,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     // the chunk's unnormalised O (relative to m_run) out of tensor memory
 #pragma unroll
     for (int d = 0; d < ND; ++d) acc[d] = 0.f;
-    if (ok && t_last >= 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[t_last & 1], (uint32_t)(t_last >> 1) & 1u));
+    if (ok && T > 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(T - 1) & 1], (uint32_t)((T - 1) >> 1) & 1u));
       if (ok) {
         tc_fence_after();
 #pragma unroll
@@ -457,32 +446,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
 
   tc_fence_before();
   __syncthreads();                       // all tiles consumed
-  // ---- the two groups' partial results (each relative to its own reference maximum) become one:
-  // group 1 hands its (O, m, l) over through shared memory (the K/V ring is free now)
-  {
-    float *gx = reinterpret_cast<float *>(sm + OFF_KV) + (size_t)gtid * (ND + 2);
-    if (row_warp && grp == 1 && T > 1) {
-#pragma unroll
-      for (int d = 0; d < ND; d += 2) *reinterpret_cast<float2 *>(gx + d) = make_float2(acc[d], acc[d + 1]);
-      *reinterpret_cast<float2 *>(gx + ND) = make_float2(m_run, l_run);
-    }
-    if (T > 1) __syncthreads();
-    if (row_warp && grp == 0 && T > 1) {
-      const float2 ml = *reinterpret_cast<const float2 *>(gx + ND);
-      const float m_new = fmaxf(m_run, ml.x);
-      const float mu = m_new == -INFINITY ? 0.f : m_new;
-      const float a = exp2f(m_run - mu), bw = exp2f(ml.x - mu);      // exp2(-inf) = 0
-#pragma unroll
-      for (int d = 0; d < ND; d += 2) {
-        const float2 o = *reinterpret_cast<const float2 *>(gx + d);
-        acc[d] = acc[d] * a + o.x * bw;
-        acc[d + 1] = acc[d + 1] * a + o.y * bw;
-      }
-      l_run = l_run * a + ml.y * bw;
-      m_run = m_new;
-    }
-    if (T > 1) __syncthreads();          // the hand-over area is part of the chunk-merge buffer below
-  }
   const bool failed = s_error != 0;
   // ---- merge over the chunks.  Every CTA receives, from every chunk j (itself included), the
   // dims [c * wc, (c + 1) * wc) of all rows plus (m, l): recv[j][row][wc + 4].
@@ -491,7 +454,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   constexpr int RR = DUP ? 64 : 128;     // rows per source chunk in the receive buffer
   float *recv = reinterpret_cast<float *>(sm + OFF_KV);
   if (P.chunks > 1) cluster_sync_all();  // the receive buffer reuses the K/V ring: every CTA of the cluster is done with its tiles
-  if (row_in && grp == 0) {
+  if (row_in) {
     const uint32_t mine = smem_u32(recv + ((size_t)c * RR + row) * rs);
 #pragma unroll
     for (int d = 0; d < ND; d += 4) {
@@ -509,7 +472,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     }
   }
   if (P.chunks > 1) cluster_sync_all(); else __syncthreads();
-  if (row_in && grp == 0 && !failed) {
+  if (row_in && !failed) {
     const int ncol = DUP ? wc / 2 : wc;                    // this thread's share of the CTA's dims
     const int col0 = DUP ? half * ncol : 0;
     float mm = -INFINITY;
@@ -547,7 +510,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       }
     }
   }
-  if (warp == MMA_WARP) {
+  if (warp == 5) {
     if (failed) {      // MMAs issued before a wait ran out may still be running: no free under them
       if (lane == 0) {
         umma_commit(&drain_bar);
