@@ -771,8 +771,7 @@ cudaError_t layer_stream(Launch L, const LayerJob &job, unsigned *sync, unsigned
     ph.sumsq = j.sumsq;
     ph.ncols = j.ncols;
     if (outs) outs[p] = SplitIn{j.Y, slots, j.split_stride, j.ldy, (unsigned)ph.ctas, ph.units, (unsigned)ph.kblocks};
-    use_count[p] += 1u;
-    ph.done_target = use_count[p] * (unsigned)grid;
+    ph.done_target = (use_count[p] + 1u) * (unsigned)grid;     // use_count advances once the launch is accepted
     ph.ready_target = ph.done_target;
     for (int i = 0; i < 3; ++i) {
       const int k = i < j.m.n ? i : 0;
@@ -801,7 +800,10 @@ cudaError_t layer_stream(Launch L, const LayerJob &job, unsigned *sync, unsigned
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   ++g_launches;
-  return cudaLaunchKernelEx(&cfg, layer_stream_kernel, Mx, P);
+  e = cudaLaunchKernelEx(&cfg, layer_stream_kernel, Mx, P);
+  if (e == cudaSuccess)
+    for (int p = 0; p < job.n_phases; ++p) use_count[p] += 1u;
+  return e;
 }
 
 }  // namespace koala

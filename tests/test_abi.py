@@ -56,3 +56,29 @@ def test_init_rejects_bad_arguments_before_touching_the_device():
     lib.koala_destroy(ctx)
     assert lib.koala_draft(None, 0) == 1 and lib.koala_verify(None, None) == 1
     assert lib.koala_gemm_bf16(None, None, None, None, 0, 0, 0, 0, None, 0, 1, 0, None, None) == 1
+
+
+def test_debug_header_symbols_are_exported_too():
+    """The diagnostic exports (tuning, launch counter, timeout self-test, workspace guards) are
+    declared outside the interface, in csrc/koala_debug.h, and exported by the same library."""
+    text = open(os.path.join(ROOT, "paper_2408_08146_b200", "csrc", "koala_debug.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = sorted(set(re.findall(r"\b(koala_[a-z0-9_]+)\s*\(", text)))
+    assert {"koala_set_tuning", "koala_launch_count", "koala_selftest_timeout", "koala_debug_check_guards"} <= set(names)
+    lib = binding.load_library()
+    for n in names:
+        assert hasattr(lib, n), f"libkoala.so does not export {n}"
+    # none of them is declared in the interface header
+    assert not set(names) & set(_declared_symbols())
+
+
+def test_token_tile_rows_of_the_standalone_multiply():
+    """koala_gemm_x_rows: whole token tiles - multiples of 16 up to 128 tokens; beyond that 256-token
+    tiles for plain operands and for pairs (which keep value and residual in one accumulator there)."""
+    lib = binding.load_library()
+    rows = lambda m, pair: int(lib.koala_gemm_x_rows(m, pair))
+    assert [rows(m, 1) for m in (1, 16, 17, 64, 100, 128)] == [16, 16, 32, 64, 112, 128]
+    assert [rows(m, 1) for m in (129, 200, 256, 257, 512)] == [144, 208, 256, 512, 512]
+    assert [rows(m, 0) for m in (10, 128, 129, 256, 300)] == [16, 128, 144, 256, 512]
+    assert rows(0, 1) == 0
+    assert int(lib.koala_gemm_static_scratch_bytes()) == 8 << 20
