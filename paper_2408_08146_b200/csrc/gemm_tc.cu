@@ -40,7 +40,8 @@ namespace {
 constexpr int BM = 128;             // weight rows per CTA (MMA M)
 constexpr int BK = 64;              // K elements per stage: 128 bytes of bf16 = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int THREADS = 192;
+constexpr int THREADS = 192;        // producer warp, MMA warp, four epilogue warps
+constexpr int THREADS_WIDE = 576;   // 256-row weight tiles: sixteen epilogue warps, four per 32 accumulator lanes
 constexpr int W_STAGE_BYTES = BM * BK * 2;
 constexpr int E_TIMEOUT = 6;
 constexpr int MAX_STAGES = 12;
@@ -79,7 +80,7 @@ __device__ __forceinline__ unsigned sk_owner(unsigned u, unsigned ctas, unsigned
   return ((u + 1u) * ctas - 1u) / units;
 }
 
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(THREADS_WIDE, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
                const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX,
                const __grid_constant__ CUtensorMap tmXlo, const TcParams P) {
@@ -137,7 +138,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&acc_full[i], 1);
-      mbar_init(&acc_empty[i], 4);       // one arrival per epilogue warp
+      mbar_init(&acc_empty[i], (blockDim.x >> 5) - 2);   // one arrival per epilogue warp
     }
     mbar_init(&drain_bar, 1);
     s_error = 0;
@@ -292,6 +293,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quarter = warp & 3;        // the 32 tensor-memory lanes this warp may read
+    // with more than four epilogue warps the warps of a lane quarter share the token columns
+    const int n_ch = ((int)(blockDim.x >> 5) - 2) >> 2;
+    const int c_per = (((P.tt >> 4) + n_ch - 1) / n_ch) << 4;
+    const int c_lo = min(((warp - 2) >> 2) * c_per, P.tt);
+    const int c_hi = min(c_lo + c_per, P.tt);
     pdl_wait();                          // the output buffer may still be read by the previous kernel
     bool ok = true;
     int seg = 0;
@@ -316,18 +322,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       const int feat = row0 + hw * BM + quarter * 32 + lane;
       float *Yp = P.Y + (size_t)slot * P.split_stride + col_off + feat;
       const uint32_t lane_base = tmem_acc + (uint32_t)((buf + hw) * P.tmem_cols) + ((uint32_t)(quarter * 32) << 16);
-      for (int c0 = 0; c0 < P.tt; c0 += 16) {
-        uint32_t v[16], w[16];
-        tmem_ld16(lane_base + (uint32_t)c0, v);
-        if (P.pair && !P.accp) tmem_ld16(lane_base + (uint32_t)(P.tt + c0), w);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      // 16 token columns per step; the next step's accumulator read is in flight while this
+      // step's values are stored
+      // (registers of a read in flight are not touched before its wait)
+      uint32_t va[16], vb[16];
+      auto store16 = [&](const uint32_t (&v)[16], int c0) {
         if (feat < n_rows) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int t = tok0 + c0 + j;
-            float r = __uint_as_float(v[j]);
-            if (P.pair && !P.accp) r += __uint_as_float(w[j]);
-            if (t < P.R) Yp[(size_t)t * P.ldy] = r;
+            if (t < P.R) Yp[(size_t)t * P.ldy] = __uint_as_float(v[j]);
+          }
+        }
+      };
+      if (P.pair && !P.accp) {
+        // value and residual rows in separate accumulator columns: added here
+        for (int c0 = c_lo; c0 < c_hi; c0 += 16) {
+          tmem_ld16(lane_base + (uint32_t)c0, va);
+          tmem_ld16(lane_base + (uint32_t)(P.tt + c0), vb);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < 16; ++j) va[j] = __float_as_uint(__uint_as_float(va[j]) + __uint_as_float(vb[j]));
+          store16(va, c0);
+        }
+      } else {
+        if (c_lo < c_hi) tmem_ld16(lane_base + (uint32_t)c_lo, va);
+        for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          const bool has_b = c0 + 16 < c_hi;
+          if (has_b) tmem_ld16(lane_base + (uint32_t)(c0 + 16), vb);
+          store16(va, c0);
+          if (has_b) {
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (c0 + 32 < c_hi) tmem_ld16(lane_base + (uint32_t)(c0 + 32), va);
+            store16(vb, c0 + 16);
           }
         }
       }
@@ -395,6 +423,8 @@ int g_tune_late_w = 0;      // 1 = weights wait for the dependency too
 int g_tune_early_stages = -1; // < 0 = all stages
 int g_tune_no_wave_split = 0; // 1 = several token tiles keep the one-wave rule's split factor
 int g_tune_no_accp = 0;      // 1 = pairs of more than 128 tokens as two 128-token tiles with extra columns
+int g_tune_epi = 0;         // 1, 2: that many epilogue warps per lane quarter for 256-row weight tiles (default 4)
+int g_tune_epi_narrow = 0;  // 1, 2, 4: epilogue warps per lane quarter for 128-row weight tiles (default by token tile)
 int g_tune_pf = 0;           // > 0: weight tiles requested into L2 ahead of the ring in that mode
 int g_tune_no_wide = 0;      // 1 = 128 weight rows per CTA also for wide token tiles
 int g_tune_traffic_div = 8; // split <= K_in / (div * tokens)
@@ -475,6 +505,8 @@ void tc_set_tuning(int key, int value) {
   if (key == 11) g_tune_no_wide = value;
   if (key == 13) g_tune_no_accp = value;
   if (key == 14) g_tune_pf = value;
+  if (key == 15) g_tune_epi = value;
+  if (key == 16) g_tune_epi_narrow = value;
   if (key == 2) g_tune_max_split = value;
   if (key == 3) g_tune_no_streamk = value;
   if (key == 5) g_tune_l2_ahead = value;
@@ -691,7 +723,15 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
     *out = SplitIn{Y, sk ? sk_slots : split, split_stride, ldy, sk ? (unsigned)sk_ctas : 0u, P.sk_units,
                    (unsigned)P.kblocks, (sk && wide) ? 1u : 0u};
   }
-  return launch_k(gemm_tc_kernel, grid, dim3(THREADS), smem, L.st, L.pdl, mw[0], mw[1], mw[2], mx, mxlo, P);
+  // Epilogue warps per 32 accumulator lanes.  256-row tiles keep one accumulator set, so the MMAs
+  // of a CTA's next tile wait for the epilogue: sixteen warps (13B-shaped verification of 256 rows:
+  // 18.3 ms with four, 16.8 with eight, 16.3 with sixteen).  128-row tiles: eight warps up to 48
+  // tokens (measured 2-3 % faster per verification and per draft pass, 8 to 48 tokens), four beyond
+  // (64 and 128 tokens measured 1-2 % slower with eight).
+  int groups = wide ? 4 : (tt <= 48 ? 2 : 1);
+  const int forced = wide ? g_tune_epi : g_tune_epi_narrow;
+  if (forced == 1 || forced == 2 || forced == 4) groups = forced;
+  return launch_k(gemm_tc_kernel, grid, dim3(64 + 128 * groups), smem, L.st, L.pdl, mw[0], mw[1], mw[2], mx, mxlo, P);
 }
 
 }  // namespace koala

@@ -26,7 +26,9 @@ extern "C" {
  * key 12 = key chunks per (sequence, head) of the tcgen05 attention kernel (0 = chosen from the shape);
  * key 13 = 1 runs pairs of more than 128 tokens as 128-token tiles with the residual rows as extra
  * accumulator columns (the form used up to 128 tokens) instead of 256-token tiles with two accumulating
- * MMAs; key 14 = weight tiles requested into L2 ahead of the ring in the 256-token form (default 0). */
+ * MMAs; key 14 = weight tiles requested into L2 ahead of the ring in the 256-token form (default 0);
+ * keys 15 (256-row weight tiles) and 16 (128-row tiles) = 1, 2 or 4: that many epilogue warps per
+ * 32 accumulator lanes instead of the default. */
 void koala_set_tuning(int key, int value);
 
 /* Kernels launched by the library in this process so far (all contexts). */
