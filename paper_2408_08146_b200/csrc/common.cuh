@@ -47,10 +47,16 @@ struct SplitIn {
   size_t stride;
   int ld;
   unsigned sk_ctas, sk_units, sk_kb;
-  unsigned sk_wide;        // stream-K: 1 = the weight tiles are 256 columns wide instead of 128
+  unsigned sk_wide;        // stream-K: weight tiles of 128 << sk_wide columns
+  // several matrices side by side whose widths are not whole tiles (0 = not the case): the columns
+  // at which the second and third matrix start, and the tiles before them
+  unsigned sk_m0, sk_m1, sk_t0, sk_t1;
   __device__ __forceinline__ int count(int c) const {
     if (sk_ctas == 0) return n;
-    const unsigned u0 = (unsigned)(c >> (7 + sk_wide)) * sk_kb;
+    const unsigned sh = 7u + sk_wide, uc = (unsigned)c;
+    unsigned tile = uc >> sh;
+    if (sk_m0 != 0 && uc >= sk_m0) tile = uc < sk_m1 ? sk_t0 + ((uc - sk_m0) >> sh) : sk_t1 + ((uc - sk_m1) >> sh);
+    const unsigned u0 = tile * sk_kb;
     const unsigned first = ((u0 + 1u) * sk_ctas - 1u) / sk_units;
     const unsigned last = ((u0 + sk_kb) * sk_ctas - 1u) / sk_units;
     return (int)(last - first) + 1;

@@ -388,6 +388,259 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
   if (threadIdx.x == 0 && s_error && P.status) atomicMax(P.status, E_TIMEOUT);
 }
 
+// ------------------------------------------------------------------------------- CTA pairs
+// More than 64 tokens as a pair of activations, two CTAs of a cluster as one MMA unit
+// (cta_group::2), token tile tt = 128 or 256.  With one CTA per tile these forms are bound by what
+// L2 delivers into shared memory (128 tokens: 48 KB per 128 weight rows and K block, three times the
+// weight bytes; 256 tokens: 96 KB per 256 weight rows).  Here a pair of CTAs owns 512 weight rows:
+// every MMA has M = 256 (128 weight rows from each CTA) and N = tt tokens, of which each CTA loads
+// only its half (value rows and residual rows).  Per CTA and stage: weight rows
+// [a*256 + rank*128, +128) for the accumulators a = 0, 1 (2 x 16 KB) and tokens [rank*tt/2, +tt/2)
+// as value and residual rows (2 x tt/2 x 128 B): 48 KB (four stages) or 64 KB (three).  With 128
+// tokens the two accumulators take 256 tensor-memory columns and there are two sets, so the
+// epilogue of one segment overlaps the MMAs of the next.  Every load of both CTAs is counted on
+// the even CTA's full barrier; that CTA's MMA thread issues for the pair and its commits arrive on
+// the empty / accumulator barriers of both CTAs; each CTA's epilogue warps read its own 128
+// accumulator lanes and arrive on the even CTA's accumulator-empty barrier.  Stream-K over the
+// clusters, one cluster per SM pair.
+constexpr int PAIR_THREADS = 576;
+constexpr int PAIR_PART_BYTES = BM * BK * 2;          // 16 KB: 128 rows of one operand part
+constexpr int PAIR_MAX_STAGES = 4;
+constexpr int PAIR_ROWS = 4 * BM;                     // weight rows per cluster tile
+
+__global__ void __launch_bounds__(PAIR_THREADS, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
+                    const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX,
+                    const __grid_constant__ CUtensorMap tmXlo, const TcParams P) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ uint64_t full_bar[PAIR_MAX_STAGES];    // used in the even CTA: both CTAs' loads of a stage landed
+  __shared__ uint64_t empty_bar[PAIR_MAX_STAGES];   // per CTA: the pair's MMAs have read this stage
+  __shared__ uint64_t acc_full[2];              // per CTA: a segment's accumulators are complete
+  __shared__ uint64_t acc_empty[2];             // used in the even CTA: both CTAs' epilogues drained them
+  __shared__ uint64_t drain_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int s_error;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();
+  const unsigned cid = blockIdx.x >> 1;                       // cluster index
+  const uint32_t raw = smem_u32(smem_raw);
+  unsigned char *tiles = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+  const int KB = P.kblocks;
+  const unsigned u_lo = (unsigned)(((unsigned long long)cid * P.sk_units) / (unsigned)P.sk_ctas);
+  const unsigned u_hi = (unsigned)(((unsigned long long)(cid + 1) * P.sk_units) / (unsigned)P.sk_ctas);
+  const int n_units = (int)(u_hi - u_lo);
+  const int n_epi = (int)(blockDim.x >> 5) - 2;
+  const int tt = P.tt;                                   // 128 or 256 tokens per tile
+  const int x_part = (tt >> 1) * BK * 2;                  // this CTA's tokens, value or residual rows
+  const int stage_bytes = 2 * PAIR_PART_BYTES + 2 * x_part;
+  const int n_stages = P.stages;
+
+  auto tile_map = [&](int tile, int &row0) -> const CUtensorMap * {
+    if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * PAIR_ROWS; return &tmW2; }
+    if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * PAIR_ROWS; return &tmW1; }
+    row0 = tile * PAIR_ROWS;
+    return &tmW0;
+  };
+  const int pre = n_units < n_stages ? n_units : n_stages;
+
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < n_stages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&acc_full[i], 1);
+      mbar_init(&acc_empty[i], (uint32_t)(2 * n_epi));
+    }
+    mbar_init(&drain_bar, 1);
+    s_error = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW0) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmXlo) : "memory");
+  }
+  if (warp == 1) {
+    // the same warp of both CTAs allocates all 512 columns in both tensor memories
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_barrier();            // both CTAs' barriers exist before anything signals them
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_acc = tmem_base_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      uint32_t full_even[PAIR_MAX_STAGES];
+      for (int s = 0; s < PAIR_MAX_STAGES; ++s) full_even[s] = cluster_addr_of(smem_u32(&full_bar[s]), 0);
+      int tile = (int)(u_lo / KB), kb = (int)(u_lo % KB), row0;
+      const CUtensorMap *tmW = tile_map(tile, row0);
+      auto load_w = [&](int s) {
+        unsigned char *dst = tiles + (size_t)s * stage_bytes;
+        if (rank == 0) mbar_expect_tx(&full_bar[s], 2u * (uint32_t)stage_bytes);
+        tma_load_2d_pair(tmW, full_even[s], dst, kb * BK, row0 + (int)rank * BM);
+        tma_load_2d_pair(tmW, full_even[s], dst + PAIR_PART_BYTES, kb * BK, row0 + 2 * BM + (int)rank * BM);
+      };
+      auto load_x = [&](int s, int kbx) {
+        unsigned char *dst = tiles + (size_t)s * stage_bytes + 2 * PAIR_PART_BYTES;
+        tma_load_2d_pair(&tmX, full_even[s], dst, kbx * BK, (int)rank * (tt >> 1));
+        tma_load_2d_pair(&tmXlo, full_even[s], dst + x_part, kbx * BK, (int)rank * (tt >> 1));
+      };
+      // the first stages' weights do not depend on the kernel before this one
+      int kb_first[PAIR_MAX_STAGES];
+      for (int it = 0; it < pre; ++it) {
+        kb_first[it] = kb;
+        load_w(it);
+        if (++kb == KB) { kb = 0; ++tile; tmW = tile_map(tile, row0); }
+      }
+      pdl_wait();
+      for (int it = 0; it < pre; ++it) load_x(it, kb_first[it]);
+      bool ok = true;
+      int s = pre % n_stages;
+      uint32_t ph = (uint32_t)(pre / n_stages) & 1u;
+      for (int it = pre; it < n_units; ++it) {
+        ok = mbar_wait(&empty_bar[s], ph ^ 1u);
+        if (!ok) break;
+        load_w(s);
+        load_x(s, kb);
+        if (++kb == KB) { kb = 0; ++tile; tmW = tile_map(tile, row0); }
+        if (++s == n_stages) { s = 0; ph ^= 1u; }
+      }
+      if (!ok) atomicExch(&s_error, 1);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (even CTA)
+    if (lane == 0 && rank == 0) {
+      // D fp32, A and B bf16, both K-major, N = tt, M = 256 over the two CTAs
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(tt >> 3) << 17) |
+                             ((uint32_t)(256 >> 4) << 24);
+      bool ok = true;
+      int seg = 0;
+      bool seg_start = true;
+      int kb = (int)(u_lo % KB), s = 0, buf = 0;
+      uint32_t ph = 0;
+      for (int it = 0; it < n_units; ++it) {
+        if (seg_start && seg >= P.nbuf) {
+          ok = mbar_wait(&acc_empty[buf], (uint32_t)((seg / P.nbuf) - 1) & 1u);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        }
+        ok = mbar_wait(&full_bar[s], ph);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t wa = smem_u32(tiles + (size_t)s * stage_bytes);
+        const uint64_t da0 = smem_desc_sw128(wa);
+        const uint64_t da1 = smem_desc_sw128(wa + PAIR_PART_BYTES);
+        const uint64_t dbh = smem_desc_sw128(wa + 2 * PAIR_PART_BYTES);
+        const uint64_t dbl = smem_desc_sw128(wa + 2 * PAIR_PART_BYTES + (uint32_t)x_part);
+        const uint32_t d0 = tmem_acc + (uint32_t)(buf * 2 * tt), d1 = d0 + (uint32_t)tt;
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; ++k) {
+          const uint32_t acc = (!seg_start || k > 0) ? 1u : 0u;
+          umma2_bf16(d0, da0 + (uint64_t)(2 * k), dbh + (uint64_t)(2 * k), idesc, acc);
+          umma2_bf16(d0, da0 + (uint64_t)(2 * k), dbl + (uint64_t)(2 * k), idesc, 1u);
+          umma2_bf16(d1, da1 + (uint64_t)(2 * k), dbh + (uint64_t)(2 * k), idesc, acc);
+          umma2_bf16(d1, da1 + (uint64_t)(2 * k), dbl + (uint64_t)(2 * k), idesc, 1u);
+        }
+        umma2_commit_to(&empty_bar[s], 3);
+        const bool seg_end = (kb == KB - 1) || it == n_units - 1;
+        if (seg_end) {
+          umma2_commit_to(&acc_full[buf], 3);
+          ++seg;
+          buf = (P.nbuf == 2) ? (buf ^ 1) : 0;
+        }
+        seg_start = seg_end;
+        if (++kb == KB) kb = 0;
+        if (++s == n_stages) { s = 0; ph ^= 1u; }
+      }
+      if (!ok) atomicExch(&s_error, 1);
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (both CTAs)
+    const int quarter = warp & 3;
+    const int n_ch = n_epi >> 2;
+    const int c_per = (((tt >> 4) + n_ch - 1) / n_ch) << 4;   // token columns in steps of 16
+    const int c_lo = min(((warp - 2) >> 2) * c_per, tt);
+    const int c_hi = min(c_lo + c_per, tt);
+    const uint32_t acc_empty_even[2] = {cluster_addr_of(smem_u32(&acc_empty[0]), 0),
+                                        cluster_addr_of(smem_u32(&acc_empty[1]), 0)};
+    bool ok = true;
+    int seg = 0;
+    unsigned u = u_lo;
+    while (u < u_hi && ok) {
+      const int tile = (int)(u / KB);
+      unsigned seg_hi = (unsigned)(tile + 1) * KB;
+      if (seg_hi > u_hi) seg_hi = u_hi;
+      const int buf = seg % P.nbuf;
+      ok = mbar_wait(&acc_full[buf], (uint32_t)(seg / P.nbuf) & 1u);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      int row0, col_off = 0, n_rows = P.n0;
+      if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * PAIR_ROWS; col_off = P.n0 + P.n1; n_rows = P.n2; }
+      else if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * PAIR_ROWS; col_off = P.n0; n_rows = P.n1; }
+      else row0 = tile * PAIR_ROWS;
+      // partial-sum slot = rank of this cluster among the tile's contributors
+      const int slot = (int)cid - (int)sk_owner((unsigned)tile * KB, (unsigned)P.sk_ctas, P.sk_units);
+      for (int a = 0; a < 2; ++a) {
+        const int feat = row0 + a * 2 * BM + (int)rank * BM + quarter * 32 + lane;
+        float *Yp = P.Y + (size_t)slot * P.split_stride + col_off + feat;
+        const uint32_t lane_base = tmem_acc + (uint32_t)((buf * 2 + a) * tt) + ((uint32_t)(quarter * 32) << 16);
+        uint32_t va[16], vb[16];
+        auto store16 = [&](const uint32_t (&v)[16], int c0) {
+          if (feat < n_rows) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int t = c0 + j;
+              if (t < P.R) Yp[(size_t)t * P.ldy] = __uint_as_float(v[j]);
+            }
+          }
+        };
+        if (c_lo < c_hi) tmem_ld16(lane_base + (uint32_t)c_lo, va);
+        for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          const bool has_b = c0 + 16 < c_hi;
+          if (has_b) tmem_ld16(lane_base + (uint32_t)(c0 + 16), vb);
+          store16(va, c0);
+          if (has_b) {
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (c0 + 32 < c_hi) tmem_ld16(lane_base + (uint32_t)(c0 + 32), va);
+            store16(vb, c0 + 16);
+          }
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(acc_empty_even[buf]);
+      ++seg;
+      u = seg_hi;
+    }
+    if (!ok) atomicExch(&s_error, 1);
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1 && rank == 0 && s_error) {
+    // a wait ran out: MMAs issued before that may still be running on both tensor memories
+    if (lane == 0) {
+      asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                   ::"r"(smem_u32(&drain_bar)) : "memory");
+      (void)mbar_wait(&drain_bar, 0);
+    }
+    __syncwarp();
+  }
+  // neither CTA frees tensor memory or leaves while the other may still be signalled or read
+  cluster_barrier();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(512u) : "memory");
+  }
+  if (threadIdx.x == 0 && s_error && P.status) atomicMax(P.status, E_TIMEOUT);
+}
+
 // ------------------------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
@@ -402,6 +655,7 @@ constexpr int MAX_DEVICES = 64;
 struct DevInfo {
   bool ready;
   int smem_optin, num_sms;
+  int pair_clusters;    // CTA pairs of gemm_tc_pair_kernel that can be resident at once (0: not usable)
 };
 DevInfo g_dev[MAX_DEVICES] = {};
 thread_local int t_dev = 0;          // the calling thread's current device as of its last use_current_device()
@@ -415,6 +669,7 @@ bool use_current_device() {
 }
 #define g_smem_optin (g_dev[t_dev].smem_optin)
 #define g_num_sms (g_dev[t_dev].num_sms)
+#define g_pair_clusters (g_dev[t_dev].pair_clusters)
 int g_tune_stages = 0;      // 0 = as many as fit (at most 8)
 int g_tune_max_split = 0;   // 0 = default rule
 int g_tune_no_streamk = 0;  // 1 = always the per-tile decomposition
@@ -425,6 +680,8 @@ int g_tune_no_wave_split = 0; // 1 = several token tiles keep the one-wave rule'
 int g_tune_no_accp = 0;      // 1 = pairs of more than 128 tokens as two 128-token tiles with extra columns
 int g_tune_epi = 0;         // 1, 2: that many epilogue warps per lane quarter for 256-row weight tiles (default 4)
 int g_tune_epi_narrow = 0;  // 1, 2, 4: epilogue warps per lane quarter for 128-row weight tiles (default by token tile)
+int g_tune_no_pair2 = 0;    // 1 = no CTA-pair kernel; 2 = not for 65 to 128 tokens
+int g_tune_pair_min = 0;    // > 0: fewest rows for the CTA-pair kernel
 int g_tune_pf = 0;           // > 0: weight tiles requested into L2 ahead of the ring in that mode
 int g_tune_no_wide = 0;      // 1 = 128 weight rows per CTA also for wide token tiles
 int g_tune_traffic_div = 8; // split <= K_in / (div * tokens)
@@ -490,6 +747,29 @@ int tc_init_driver(char *err, size_t errlen) {
     snprintf(err, errlen, "cannot raise the GEMM kernel's shared memory: %s", cudaGetErrorString(e));
     return 1;
   }
+  // the CTA-pair kernel: shared-memory opt-in, and how many pairs fit on this device at once
+  {
+    const size_t smem = (size_t)3 * (2 * PAIR_PART_BYTES + 256 * BK * 2) + 1024;   // = four stages of the 128-token form
+    d.pair_clusters = 0;
+    if ((size_t)d.smem_optin >= smem + 1024 &&
+        cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(2 * (d.num_sms / 2));
+      cfg.blockDim = dim3(PAIR_THREADS);
+      cfg.dynamicSmemBytes = smem;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair_kernel, &cfg) == cudaSuccess && n > 0)
+        d.pair_clusters = n < d.num_sms / 2 ? n : d.num_sms / 2;
+      (void)cudaGetLastError();
+    }
+  }
   d.ready = true;
   g_dev[dev] = d;
   return 0;
@@ -507,6 +787,8 @@ void tc_set_tuning(int key, int value) {
   if (key == 14) g_tune_pf = value;
   if (key == 15) g_tune_epi = value;
   if (key == 16) g_tune_epi_narrow = value;
+  if (key == 17) g_tune_no_pair2 = value;
+  if (key == 18) g_tune_pair_min = value;
   if (key == 2) g_tune_max_split = value;
   if (key == 3) g_tune_no_streamk = value;
   if (key == 5) g_tune_l2_ahead = value;
@@ -629,6 +911,81 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   // two CTAs per SM measured 6-7 % faster than 256 rows with one: 7B verify 5.7 against 6.1 ms.)
   bool wide = !g_tune_no_wide && accp && bn == 256 && g_smem_optin - 2048 >= 2 * (2 * W_STAGE_BYTES + x_bytes);
   for (int i = 0; i < m.n && wide; ++i) wide = (m.n_out[i] % (2 * BM)) == 0;
+  // CTA pairs (512 weight rows per cluster, each CTA loading half of the tokens): 113 to 256 tokens
+  // as a pair, stream-K over the clusters that fit on the device at once.  The last tile of a
+  // matrix may be ragged (rows beyond the matrix are zero-filled by the loads and not stored).
+  // Measured per verification, 7B shapes: 128 rows 5.67-5.85 against 5.78-5.90 ms, 2 x 64 rows
+  // 5.50-5.85 against 5.76-5.90; the 128-token tile costs more than it saves below that (100 rows
+  // 5.53 against 5.43, 80 rows 5.25 against 4.48, where the one-CTA form uses an 80-token tile).
+  const int pair_min_rows = g_tune_pair_min > 0 ? g_tune_pair_min : 113;
+  if (pair && R >= pair_min_rows && R <= 256 && !(g_tune_no_pair2 & 1) && g_pair_clusters > 0 && split == 0 &&
+      out != nullptr && max_slots >= 2 && m.n <= 3 && (R > 128 || !(g_tune_no_pair2 & 2))) {
+    const int q0 = (m.n_out[0] + PAIR_ROWS - 1) / PAIR_ROWS, q1 = m.n > 1 ? (m.n_out[1] + PAIR_ROWS - 1) / PAIR_ROWS : 0,
+              q2 = m.n > 2 ? (m.n_out[2] + PAIR_ROWS - 1) / PAIR_ROWS : 0;
+    const int n_tiles = q0 + q1 + q2, KB = K_in / BK;
+    const long long units = (long long)n_tiles * KB;
+    long long g = g_pair_clusters;
+    if (g > units / 8) g = units / 8;
+    if (g < 1) g = 1;
+    auto slots_of = [&](long long gg) {
+      const long long per = units / gg;
+      return (int)((KB + per - 1) / per) + ((units % gg) || (KB % per) ? 1 : 0);
+    };
+    while (g > 1 && slots_of(g) > max_slots) --g;
+    if (slots_of(g) <= max_slots) {
+      const int ptt = R > 128 ? 256 : 128;
+      P.tt = ptt;
+      P.bn = ptt;
+      P.nbuf = ptt == 128 ? 2 : 1;
+      P.stages = ptt == 128 ? 4 : 3;
+      P.tiles0 = q0;
+      P.tiles1 = q0 + q1;
+      P.n0 = m.n_out[0];
+      P.n1 = m.n > 1 ? m.n_out[1] : 0;
+      P.n2 = m.n > 2 ? m.n_out[2] : 0;
+      P.kblocks = KB;
+      P.sk_ctas = (int)g;
+      P.sk_units = (unsigned)units;
+      P.split = 1;
+      P.split_stride = split_stride;
+      P.status = status;
+      CUtensorMap mw[3], mx, mxlo;
+      for (int i = 0; i < 3; ++i) {
+        const int j = i < m.n ? i : 0;
+        if (!get_map(m.W[j], m.n_out[j], K_in, BM, &mw[i])) return cudaErrorInvalidValue;
+      }
+      if (!get_map(X.hi, x_rows_alloc, K_in, ptt / 2, &mx)) return cudaErrorInvalidValue;
+      if (!get_map(X.lo, x_rows_alloc, K_in, ptt / 2, &mxlo)) return cudaErrorInvalidValue;
+      SplitIn si{Y, slots_of(g), split_stride, ldy, (unsigned)g, (unsigned)units, (unsigned)KB, 2u};
+      bool ragged = false;
+      for (int i = 0; i + 1 < m.n; ++i) ragged = ragged || (m.n_out[i] % PAIR_ROWS) != 0;
+      if (ragged) {
+        si.sk_m0 = (unsigned)P.n0;
+        si.sk_m1 = m.n > 2 ? (unsigned)(P.n0 + P.n1) : 0xFFFFFFFFu;
+        si.sk_t0 = (unsigned)q0;
+        si.sk_t1 = (unsigned)(q0 + q1);
+      }
+      *out = si;
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)(2 * g));
+      cfg.blockDim = dim3(PAIR_THREADS);
+      cfg.dynamicSmemBytes = (size_t)P.stages * (2 * PAIR_PART_BYTES + ptt * BK * 2) + 1024;
+      cfg.stream = L.st;
+      cudaLaunchAttribute attr[2];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = L.pdl ? 1 : 0;
+      attr[1].id = cudaLaunchAttributeClusterDimension;
+      attr[1].val.clusterDim.x = 2;
+      attr[1].val.clusterDim.y = 1;
+      attr[1].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 2;
+      ++g_launches;
+      return cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel, mw[0], mw[1], mw[2], mx, mxlo, P);
+    }
+    memset(&P, 0, sizeof(P));
+    P.tt = tt; P.pair = pair; P.accp = accp; P.ztiles = ztiles; P.Y = Y; P.ldy = ldy; P.R = R; P.bn = bn; P.tmem_cols = cols;
+  }
   const int bmw = wide ? 2 * BM : BM;
   P.wide = wide ? 1 : 0;
   const int t0 = (m.n_out[0] + bmw - 1) / bmw;

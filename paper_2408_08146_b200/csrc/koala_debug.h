@@ -28,7 +28,8 @@ extern "C" {
  * accumulator columns (the form used up to 128 tokens) instead of 256-token tiles with two accumulating
  * MMAs; key 14 = weight tiles requested into L2 ahead of the ring in the 256-token form (default 0);
  * keys 15 (256-row weight tiles) and 16 (128-row tiles) = 1, 2 or 4: that many epilogue warps per
- * 32 accumulator lanes instead of the default. */
+ * 32 accumulator lanes instead of the default; key 17 = 1: no CTA-pair GEMM kernel, 2: not up to 128
+ * rows; key 18 = fewest rows for it (default 113). */
 void koala_set_tuning(int key, int value);
 
 /* Kernels launched by the library in this process so far (all contexts). */
