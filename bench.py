@@ -384,7 +384,8 @@ def run_koala(args):
                 "tokens": int(n[1]), "schedule": "the timed region's slice, replayed from the same context lengths",
                 "h2d_bytes_per_step": 4 * cfg.B, "d2h_bytes_per_step": 4 * cfg.B * (eng.out_stride + 1)},
         "gpu_launches": int(n[2]),
-        "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel (all weight-streaming GEMMs of a step)",
+        "roofline": {"bound": "hbm", "kernel": "gemm_tc_pair_kernel + gemm_tc_kernel (all weight-streaming GEMMs of a step: the CTA-pair form "
+                               "for the verification's 256 rows, the one-CTA form for the draft passes and the LM head)",
                      "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                      "peak_source": f"of {peaks['source']}", "traffic": None,
                      "traffic_source": "not captured for the current kernel in this run (see the ncu summaries under profiles/)",
