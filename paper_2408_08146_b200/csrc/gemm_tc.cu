@@ -916,7 +916,9 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   // matrix may be ragged (rows beyond the matrix are zero-filled by the loads and not stored).
   // Measured per verification, 7B shapes: 128 rows 5.67-5.85 against 5.78-5.90 ms, 2 x 64 rows
   // 5.50-5.85 against 5.76-5.90; the 128-token tile costs more than it saves below that (100 rows
-  // 5.53 against 5.43, 80 rows 5.25 against 4.48, where the one-CTA form uses an 80-token tile).
+  // 5.53 against 5.43, 80 rows 5.25 against 4.48, where the one-CTA form uses an 80-token tile;
+  // with 32- and 64-token tiles the pair form measured 13-15 % slower at 16 to 64 rows, where two
+  // independent CTAs per SM overlap each other's start and end).
   const int pair_min_rows = g_tune_pair_min > 0 ? g_tune_pair_min : 113;
   if (pair && R >= pair_min_rows && R <= 256 && !(g_tune_no_pair2 & 1) && g_pair_clusters > 0 && split == 0 &&
       out != nullptr && max_slots >= 2 && m.n <= 3 && (R > 128 || !(g_tune_no_pair2 & 2))) {
