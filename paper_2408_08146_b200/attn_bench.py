@@ -37,11 +37,14 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--mma-sync", action="store_true")
     ap.add_argument("--chunks", type=int, default=0, help="key chunks per (sequence, head): 1, 2, 4, 8; 0 = automatic")
+    ap.add_argument("--l2-ahead", type=int, default=-1, help="K/V tiles requested into L2 ahead of the ring (-1 = the library's default)")
     args = ap.parse_args()
     lib = binding.load_library()
     if args.mma_sync:
         lib.koala_set_tuning(9, 1 << 20)
     lib.koala_set_tuning(12, args.chunks)
+    if args.l2_ahead >= 0:
+        lib.koala_set_tuning(19, args.l2_ahead)
     n = args.rows
     cfg = reduced(T7_EAGLE, 2, K=1, N=n, B=args.batch, D=min(5, max(1, n - 1)), V=4096,
                   S_max=((args.context + n + 127) // 128) * 128)

@@ -38,7 +38,8 @@ namespace {
 
 constexpr int DH = 128;
 constexpr int TK = 64;                       // keys per tile
-constexpr int NKV = 3;                       // K/V stages
+constexpr int NKV = 3;                       // K/V stages (four with at most 64 rows, where Q takes half the room)
+constexpr int NKV_MAX = 4;
 constexpr int SUB = 64 * 64 * 2;             // one [64 keys][64 dims] block: 8 KB
 constexpr int QSUB = 128 * 64 * 2;           // one [128 rows][64 columns] block: 16 KB
 constexpr int OFF_Q = 0;                     // Q hi (2 blocks), Q lo (2 blocks)
@@ -119,23 +120,32 @@ struct AttnParams {
   bf16 *out, *out_lo;      // [R][n_heads * 128]
   int rows_per_seq, n_heads, S_max, chunks;
   int longest_first;       // 1: grid slot y / n_heads takes the sequence with that rank in descending cache length
+  int l2_ahead;            // K/V tiles requested into L2 this many tiles ahead of the ring (0 = none)
+  int dry_pass;            // 1: the row warps make a dry pass over the tile loop body before the dependency wait
   int *status;
 };
 
-// DUP (at most 64 query rows): the rows are loaded twice, into MMA rows r and r + 64, so that all
-// four row warps work: warps 0,1 take the first 32 keys of every tile and the first 64 output
-// dims of rows 0..63, warps 2,3 the other halves of the same rows (tile row maxima are exchanged
-// through shared memory).  Otherwise warp w owns rows 32w .. 32w+31 entirely.
+// DUP (at most 64 query rows): the MMA's 128 rows hold both parts of the operand pair (of Q for S,
+// of P for P V), so that one pass of MMAs gives both partial products, to be added: warp w owns
+// queries 16w .. 16w+15, whose value parts are MMA rows (= tensor-memory lanes) 32w .. 32w+15 and
+// whose residual parts are rows 32w+16 .. 32w+31.  Lanes l and l+16 of a warp therefore hold the
+// two partial scores S_v, S_r of one query: they swap halves by shuffles (no shared memory, no
+// barrier), after which lane l has S = S_v + S_r for keys 0..31 of the tile and lane l+16 for keys
+// 32..63; the row maximum is one more shuffle; at the end they swap halves of O_v, O_r the same
+// way and write dims 0..63 and 64..127.  Otherwise warp w owns rows 32w .. 32w+31 entirely and
+// the pair is two accumulating MMAs.
 template <bool DUP>
 __global__ void __launch_bounds__(THREADS, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_constant__ CUtensorMap tmQl,
                     const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const AttnParams P) {
-  constexpr int NC = DUP ? 32 : 64;      // score columns (keys of a tile) per thread
+  constexpr int NC = DUP ? 32 : 64;      // keys of a tile per thread
   constexpr int ND = DUP ? 64 : 128;     // output dims per thread
+  constexpr int PB = DUP ? QSUB : P_BUF; // bytes of one P buffer
+  constexpr int NST = DUP ? NKV + 1 : NKV;             // K/V stages
+  constexpr int OKV = DUP ? OFF_KV - KV_STAGE : OFF_KV; // the ring starts where the second half of Q would be
   extern __shared__ unsigned char smem_raw[];
-  __shared__ uint64_t q_full, kv_full[NKV], kv_empty[NKV], s_full[2], p_full[2], pv_done[2], x_bar[2], drain_bar;
-  __shared__ float xch[2][128];
+  __shared__ uint64_t q_full, kv_full[NKV_MAX], kv_empty[NKV_MAX], s_full[2], p_full[2], pv_done[2], drain_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int s_error;
 
@@ -147,19 +157,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   int b = blockIdx.y / P.n_heads;
   const int h = blockIdx.y % P.n_heads;
   const int H = P.n_heads * DH;
-  const int n_q = (P.rows_per_seq + 31) >> 5;             // 32-row groups in use
-  const int n_arrive = DUP ? 2 * n_q : n_q;               // row warps in use
+  const int n_q = DUP ? (P.rows_per_seq + 15) >> 4 : (P.rows_per_seq + 31) >> 5;   // row warps in use (16 or 32 queries each)
+  const int n_arrive = n_q;
 
   pdl_launch_dependents();
   if (threadIdx.x == 0) {
     mbar_init(&q_full, 1);
-    for (int s = 0; s < NKV; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+    for (int s = 0; s < NST; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
     mbar_init(&drain_bar, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s_full[i], 1);
       mbar_init(&p_full[i], (uint32_t)n_arrive);
       mbar_init(&pv_done[i], 1);
-      mbar_init(&x_bar[i], 2);
     }
     s_error = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -179,49 +188,67 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   tc_fence_after();
   const uint32_t tmem = tmem_base_slot;
 
-  pdl_wait();                      // Q, the tree rows of K/V and the row plan come from earlier kernels
-  if (P.longest_first) {
-    // More CTAs than SMs: the CTAs beyond the first round start when the first ones finish, so the
-    // sequences are taken longest first and the late CTAs belong to the shortest one.  Lane l holds
-    // sequence l's length; its rank is the number of sequences that are longer (ties: lower index).
-    const int nb = (int)gridDim.y / P.n_heads;              // <= 32 here
-    const int len_l = lane < nb ? P.plan.kv_len[lane] : -1;
-    int rank = 0;
-    for (int j = 0; j < nb; ++j) {
-      const int len_j = __shfl_sync(0xffffffffu, len_l, j);
-      rank += (len_j > len_l || (len_j == len_l && j < lane)) ? 1 : 0;
+  // Q, the tree rows of K/V and the row plan come from earlier kernels: everything that reads them
+  // comes after the dependency wait in read_plan().  The row warps call it inside their tile loop,
+  // after a dry pass over the loop body (see there); the other threads here.
+  int ctx = 0, kv_len = 0, tile_lo = 0, T = 0;
+  auto read_plan = [&]() {
+    pdl_wait();
+    if (P.longest_first) {
+      // More CTAs than SMs: the CTAs beyond the first round start when the first ones finish, so the
+      // sequences are taken longest first and the late CTAs belong to the shortest one.  Lane l holds
+      // sequence l's length; its rank is the number of sequences that are longer (ties: lower index).
+      const int nb = (int)gridDim.y / P.n_heads;              // <= 32 here
+      const int len_l = lane < nb ? P.plan.kv_len[lane] : -1;
+      int rank = 0;
+      for (int j = 0; j < nb; ++j) {
+        const int len_j = __shfl_sync(0xffffffffu, len_l, j);
+        rank += (len_j > len_l || (len_j == len_l && j < lane)) ? 1 : 0;
+      }
+      const unsigned hit = __ballot_sync(0xffffffffu, lane < nb && rank == b);
+      b = hit ? __ffs(hit) - 1 : b;
     }
-    const unsigned hit = __ballot_sync(0xffffffffu, lane < nb && rank == b);
-    b = hit ? __ffs(hit) - 1 : b;
-  }
+    ctx = P.plan.ctx_len[b];
+    kv_len = P.plan.kv_len[b];
+    kv_len = kv_len > P.S_max ? P.S_max : kv_len;
+    const int n_tiles = (kv_len + TK - 1) / TK;
+    tile_lo = (int)(((long long)n_tiles * c) / P.chunks);
+    const int tile_hi = (int)(((long long)n_tiles * (c + 1)) / P.chunks);
+    T = tile_hi - tile_lo;
+  };
+  // row ownership of warps 0..3
+  const int half = DUP ? (lane >> 4) : 0;                   // DUP: residual lane; takes the second half of the keys / dims
+  const int row = DUP ? warp * 16 + (lane & 15) : warp * 32 + lane;
+  const bool row_warp = warp < 4 && warp < n_q;
+  const bool row_in = row_warp && row < P.rows_per_seq;
+  if (!row_warp) read_plan();
   if (threadIdx.x == 128) {        // warp 4 lane 0: the queries do not depend on the plan
-    mbar_expect_tx(&q_full, (uint32_t)(4 * QSUB));
-#pragma unroll
-    for (int part = 0; part < 2; ++part)
+    if (DUP) {
+      // of every 32 MMA rows the first 16 are the values of 16 queries, the other 16 their residuals
+      mbar_expect_tx(&q_full, (uint32_t)(2 * QSUB));
 #pragma unroll
       for (int hb = 0; hb < 2; ++hb)
 #pragma unroll
-        for (int rh = 0; rh < 2; ++rh)
-          tma_load_2d(part ? &tmQl : &tmQh, &q_full, sm + OFF_Q + (part * 2 + hb) * QSUB + rh * (QSUB / 2),
-                      h * DH + 64 * hb, b * P.rows_per_seq + (DUP ? 0 : 64 * rh));
+        for (int g = 0; g < 4; ++g)
+#pragma unroll
+          for (int part = 0; part < 2; ++part)
+            tma_load_2d(part ? &tmQl : &tmQh, &q_full, sm + OFF_Q + hb * QSUB + (32 * g + 16 * part) * 128,
+                        h * DH + 64 * hb, b * P.rows_per_seq + 16 * g);
+    } else {
+      mbar_expect_tx(&q_full, (uint32_t)(4 * QSUB));
+#pragma unroll
+      for (int part = 0; part < 2; ++part)
+#pragma unroll
+        for (int hb = 0; hb < 2; ++hb)
+#pragma unroll
+          for (int rh = 0; rh < 2; ++rh)
+            tma_load_2d(part ? &tmQl : &tmQh, &q_full, sm + OFF_Q + (part * 2 + hb) * QSUB + rh * (QSUB / 2),
+                        h * DH + 64 * hb, b * P.rows_per_seq + 64 * rh);
+    }
   }
-  const int ctx = P.plan.ctx_len[b];
-  int kv_len = P.plan.kv_len[b];
-  kv_len = kv_len > P.S_max ? P.S_max : kv_len;
-  const int n_tiles = (kv_len + TK - 1) / TK;
-  const int tile_lo = (int)(((long long)n_tiles * c) / P.chunks);
-  const int tile_hi = (int)(((long long)n_tiles * (c + 1)) / P.chunks);
-  const int T = tile_hi - tile_lo;
-
-  // row ownership of warps 0..3
-  const int rq = DUP ? (warp & 1) : warp;                   // 32-row group
-  const int half = DUP ? (warp >> 1) : 0;                   // which half of the keys / dims
-  const int row = rq * 32 + lane;
-  const bool row_warp = warp < 4 && rq < n_q;
-  const bool row_in = row_warp && row < P.rows_per_seq;
-  const int r_glob = b * P.rows_per_seq + (row_in ? row : 0);
-  float acc[ND];
+  int r_glob = 0;
   float m_run = -INFINITY, l_run = 0.f;
+  bool have_o = false;             // this warp's O in tensor memory is complete (warp-uniform)
 
   if (warp == 4) {
     // ------------------------------------------------------------------ TMA producer
@@ -229,14 +256,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       const int y0 = (b * P.n_heads + h) * P.S_max;
       bool ok = true;
       int issued = 0;
+      auto request_l2 = [&](int t) {
+        const int y = y0 + (tile_lo + t) * TK;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+                       ::"l"(q < 2 ? &tmK : &tmV), "r"(64 * (q & 1)), "r"(y) : "memory");
+      };
+      // the cache is streamed from HBM by one CTA with a few tiles in flight: tiles beyond the ring
+      // are requested into L2 so that the ring's own loads find them there
+      for (int t = NST; t < NST + P.l2_ahead && t < T; ++t) request_l2(t);
       for (int t = 0; t < T; ++t) {
-        const int s = t % NKV;
-        if (t >= NKV) {
-          ok = mbar_wait(&kv_empty[s], (uint32_t)((t / NKV) - 1) & 1u);
+        const int s = t % NST;
+        if (P.l2_ahead > 0 && t + NST + P.l2_ahead < T) request_l2(t + NST + P.l2_ahead);
+        if (t >= NST) {
+          ok = mbar_wait(&kv_empty[s], (uint32_t)((t / NST) - 1) & 1u);
           if (!ok) break;
         }
         mbar_expect_tx(&kv_full[s], (uint32_t)KV_STAGE);
-        unsigned char *dst = sm + OFF_KV + s * KV_STAGE;
+        unsigned char *dst = sm + OKV + s * KV_STAGE;
         const int y = y0 + (tile_lo + t) * TK;
         tma_load_2d(&tmK, &kv_full[s], dst, 0, y);
         tma_load_2d(&tmK, &kv_full[s], dst + SUB, 64, y);
@@ -247,8 +285,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       if (!ok) {
         atomicExch(&s_error, 1);
         // let the copies already requested land before the block's memory goes away
-        for (int t = issued > NKV ? issued - NKV : 0; t < issued; ++t)
-          (void)mbar_wait(&kv_full[t % NKV], (uint32_t)(t / NKV) & 1u);
+        for (int t = issued > NST ? issued - NST : 0; t < issued; ++t)
+          (void)mbar_wait(&kv_full[t % NST], (uint32_t)(t / NST) & 1u);
       }
       if (T == 0 || !ok) (void)mbar_wait(&q_full, 0);      // nobody else waits for Q then
     }
@@ -260,16 +298,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) |
                                ((128u >> 4) << 24);
       auto issue_s = [&](int t) -> bool {
-        const int s = t % NKV;
-        if (!mbar_wait(&kv_full[s], (uint32_t)(t / NKV) & 1u)) return false;
+        const int s = t % NST;
+        if (!mbar_wait(&kv_full[s], (uint32_t)(t / NST) & 1u)) return false;
         tc_fence_after();
-        const uint32_t kb = sb + OFF_KV + s * KV_STAGE;
+        const uint32_t kb = sb + OKV + s * KV_STAGE;
         const uint32_t d = tmem + (uint32_t)(COL_S + (t & 1) * TK);
 #pragma unroll
-        for (int part = 0; part < 2; ++part) {            // Q value, then Q residual
+        for (int part = 0; part < (DUP ? 1 : 2); ++part) { // Q value, then Q residual (DUP: both in one operand)
 #pragma unroll
           for (int hb = 0; hb < 2; ++hb) {                 // 64-dim block
-            const uint64_t da = smem_desc_sw128(sb + OFF_Q + (part * 2 + hb) * QSUB);
+            const uint64_t da = smem_desc_sw128(sb + OFF_Q + (DUP ? hb : part * 2 + hb) * QSUB);
             const uint64_t db = smem_desc_sw128(kb + hb * SUB);
 #pragma unroll
             for (int k = 0; k < 4; ++k)
@@ -286,11 +324,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         ok = mbar_wait(&p_full[t & 1], (uint32_t)(t >> 1) & 1u);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t vb = sb + OFF_KV + (t % NKV) * KV_STAGE + 2 * SUB;
-        const uint32_t pb = sb + OFF_P + (t & 1) * P_BUF;
+        const uint32_t vb = sb + OKV + (t % NST) * KV_STAGE + 2 * SUB;
+        const uint32_t pb = sb + OFF_P + (t & 1) * PB;
         const uint32_t d = tmem + (uint32_t)COL_O;
 #pragma unroll
-        for (int part = 0; part < 2; ++part) {            // P value, then P residual
+        for (int part = 0; part < (DUP ? 1 : 2); ++part) { // P value, then P residual (DUP: both in one operand)
           const uint64_t da = smem_desc_sw128(pb + part * QSUB);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {                    // 16 keys per MMA
@@ -298,7 +336,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
             umma_bf16(d, da + (uint64_t)(2 * k), db, idesc_o, (t | part | k) ? 1u : 0u);   // O accumulates over the tiles
           }
         }
-        umma_commit(&kv_empty[t % NKV]);
+        umma_commit(&kv_empty[t % NST]);
         umma_commit(&pv_done[t & 1]);
       }
       if (!ok) atomicExch(&s_error, 1);
@@ -310,26 +348,55 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     // by more than RESCALE_STEP (then the row's O and l are multiplied by 2^(old - new) in place);
     // in between the probabilities may exceed 1 (by at most 2^RESCALE_STEP), which costs nothing in
     // fp32 / bf16-pair arithmetic, and the rows never wait for P V except to reuse a P buffer.
-    const int slot = P.plan.slot[r_glob];
-    const bool ok_row = row_in && slot >= 0;
-    const uint64_t mk0 = ok_row ? P.plan.mask[(size_t)r_glob * 2] : 0ull;
-    const uint64_t mk1 = ok_row ? P.plan.mask[(size_t)r_glob * 2 + 1] : 0ull;
+    bool ok_row = false;
+    uint64_t mk0 = 0ull, mk1 = 0ull;
     const float sc = 0.08838834764831845f * 1.4426950408889634f;    // 1/sqrt(128) * log2(e)
     const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;          // this warp's 32 TMEM lanes
-    const uint32_t prow = (uint32_t)(row * 128);
+    const uint32_t prow = (uint32_t)((DUP ? warp * 32 + (lane & 15) : row) * 128);   // this query's (value) row of the P operand
     const uint32_t psw = (uint32_t)(row & 7);
-    const uint32_t o_base = tmem + lane_sel + (uint32_t)(COL_O + ND * half);
+    const uint32_t o_base = tmem + lane_sel + (uint32_t)COL_O;     // all 128 dims of this thread's lane
     bool ok = true;
 
-    for (int t = 0; t < T; ++t) {
-      ok = __all_sync(0xffffffffu, mbar_wait(&s_full[t & 1], (uint32_t)(t >> 1) & 1u));   // warp-uniform
-      if (!ok) break;
+    // Pass t = -1 is a dry pass over the loop body, made before the dependency wait while the kernel
+    // before this one still runs: no waits, no row visible (every probability is 0), nothing handed
+    // to the MMA warp.  The body is some 20 KB of instructions that run a few times per launch; the
+    // dry pass takes their first, slow fetch off the path between the arrival of S and the first P.
+    int T_run = 1;
+    for (int t = P.dry_pass ? -1 : 0; t < T_run; ++t) {
+      if (t == 0) {
+        read_plan();
+        T_run = T;
+        if (T == 0) break;
+        r_glob = b * P.rows_per_seq + (row_in ? row : 0);
+        ok_row = row_in && P.plan.slot[r_glob] >= 0;
+        mk0 = ok_row ? P.plan.mask[(size_t)r_glob * 2] : 0ull;
+        mk1 = ok_row ? P.plan.mask[(size_t)r_glob * 2 + 1] : 0ull;
+      }
+      const bool live = t >= 0;
+      if (live) {
+        ok = __all_sync(0xffffffffu, mbar_wait(&s_full[t & 1], (uint32_t)(t >> 1) & 1u));   // warp-uniform
+        if (!ok) break;
+      }
       tc_fence_after();
       uint32_t v[NC];
-      const uint32_t base = tmem + lane_sel + (uint32_t)(COL_S + (t & 1) * TK + NC * half);
+      const uint32_t base = tmem + lane_sel + (uint32_t)(COL_S + (t & 1) * TK);
+      if constexpr (DUP) {
+        // this lane holds one part (value or residual) of the query's 64 raw scores: keep the part of
+        // this lane's 32 keys, hand the other 32 to the query's second lane, add what it hands back
+        uint32_t raw[TK];
 #pragma unroll
-      for (int c0 = 0; c0 < NC; c0 += 16) tmem_ld16(base + (uint32_t)c0, v + c0);
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        for (int c0 = 0; c0 < TK; c0 += 16) tmem_ld16(base + (uint32_t)c0, raw + c0);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float got = __shfl_xor_sync(0xffffffffu, __uint_as_float(half ? raw[j] : raw[32 + j]), 16);
+          v[j] = __float_as_uint(__uint_as_float(half ? raw[32 + j] : raw[j]) + got);
+        }
+      } else {
+#pragma unroll
+        for (int c0 = 0; c0 < NC; c0 += 16) tmem_ld16(base + (uint32_t)c0, v + c0);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      }
       const int key0 = (tile_lo + t) * TK;
       if (kv_len - key0 < TK) {
         // The last tile reaches past kv_len: those cache slots were never written and may hold
@@ -337,7 +404,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         // the value rows from kv_len on (a row is 128 bytes of each 64-dim block; the swizzle
         // only permutes inside the row).  The tile has landed: S, which this warp waited for, was
         // issued after it.  Every row warp in use writes the same zeros.
-        const uint32_t vb = sb + OFF_KV + (t % NKV) * KV_STAGE + 2 * SUB;
+        const uint32_t vb = sb + OKV + (t % NST) * KV_STAGE + 2 * SUB;
         for (int kr = kv_len - key0 + lane; kr < TK; kr += 32) {
 #pragma unroll
           for (int blk = 0; blk < 2; ++blk)
@@ -354,16 +421,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         v[j] = __float_as_uint(s);
         m_t = fmaxf(m_t, s);
       }
-      if (DUP) {
-        // the row's maximum over the whole tile: exchange with the thread that holds the other 32 keys
-        // (both threads of a row then keep the same reference maximum)
-        xch[t & 1][threadIdx.x] = m_t;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&x_bar[rq]);
-        ok = __all_sync(0xffffffffu, mbar_wait(&x_bar[rq], (uint32_t)t & 1u));
-        if (!ok) break;
-        m_t = fmaxf(m_t, xch[t & 1][threadIdx.x ^ 64]);
-      }
+      if (DUP) m_t = fmaxf(m_t, __shfl_xor_sync(0xffffffffu, m_t, 16));   // over all 64 keys: both lanes keep the same reference
       // raise the reference maximum?  (the first visible key sets it; O holds nothing of this row yet then)
       float factor = 1.f;
       if (m_t > m_run + RESCALE_STEP || (m_run == -INFINITY && m_t > -INFINITY)) {
@@ -377,8 +435,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(t - 1) & 1], (uint32_t)((t - 1) >> 1) & 1u));
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int c0 = 0; c0 < ND; c0 += 16) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < DH; c0 += 16) {          // rare: kept short
           uint32_t o[16];
           tmem_ld16(o_base + (uint32_t)c0, o);
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -398,7 +456,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       }
       const float mu = m_run == -INFINITY ? 0.f : m_run;
       float l_t = 0.f;
-      const uint32_t pb = sb + OFF_P + (uint32_t)((t & 1) * P_BUF) + prow;
+      const uint32_t pb = sb + OFF_P + (uint32_t)((t & 1) * PB) + prow;
 #pragma unroll
       for (int ch = 0; ch < NC / 8; ++ch) {
         uint32_t hi[4], lo[4];
@@ -411,36 +469,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
         }
         const uint32_t off = (((uint32_t)(ch + (NC / 8) * half)) ^ psw) << 4;
         st_shared_v4(pb + off, hi[0], hi[1], hi[2], hi[3]);
-        st_shared_v4(pb + QSUB + off, lo[0], lo[1], lo[2], lo[3]);
-        if (DUP) {                       // the copy of this row in the upper half of the MMA's rows
-          st_shared_v4(pb + 64 * 128 + off, hi[0], hi[1], hi[2], hi[3]);
-          st_shared_v4(pb + QSUB + 64 * 128 + off, lo[0], lo[1], lo[2], lo[3]);
-        }
+        // the residuals: 16 rows further down in the same operand (DUP) or the second operand
+        st_shared_v4(pb + (DUP ? 16 * 128 : QSUB) + off, lo[0], lo[1], lo[2], lo[3]);
       }
       l_run += l_t;
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full[t & 1]);
+      if (live && lane == 0) mbar_arrive(&p_full[t & 1]);
     }
-    // the chunk's unnormalised O (relative to m_run) out of tensor memory
-#pragma unroll
-    for (int d = 0; d < ND; ++d) acc[d] = 0.f;
-    if (ok && T > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(T - 1) & 1], (uint32_t)((T - 1) >> 1) & 1u));
-      if (ok) {
-        tc_fence_after();
-#pragma unroll
-        for (int c0 = 0; c0 < ND; c0 += 32) {
-          uint32_t o[32];
-          tmem_ld16(o_base + (uint32_t)c0, o);
-          tmem_ld16(o_base + (uint32_t)(c0 + 16), o + 16);
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-          for (int j = 0; j < 32; ++j) acc[c0 + j] = __uint_as_float(o[j]);
-        }
-      }
-    }
+    // every P V of the chunk has landed in tensor memory before O is read below
+    if (ok && T > 0) ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(T - 1) & 1], (uint32_t)((T - 1) >> 1) & 1u));
+    have_o = ok && T > 0;
     if (!ok) atomicExch(&s_error, 1);
   }
 
@@ -448,66 +488,101 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   __syncthreads();                       // all tiles consumed
   const bool failed = s_error != 0;
   // ---- merge over the chunks.  Every CTA receives, from every chunk j (itself included), the
-  // dims [c * wc, (c + 1) * wc) of all rows plus (m, l): recv[j][row][wc + 4].
+  // dims [c * wc, (c + 1) * wc) of all rows plus (m, l): recv[j][row][wc + 4].  The code from here
+  // on runs once per CTA, so it is written as short loops rather than unrolled over the 128 dims.
   const int wc = DH / P.chunks;
   const int rs = wc + 4;                 // floats per received row: wc dims, m, l (first keys), l (other keys), pad
   constexpr int RR = DUP ? 64 : 128;     // rows per source chunk in the receive buffer
-  float *recv = reinterpret_cast<float *>(sm + OFF_KV);
+  float *recv = reinterpret_cast<float *>(sm + OKV);
   if (P.chunks > 1) cluster_sync_all();  // the receive buffer reuses the K/V ring: every CTA of the cluster is done with its tiles
-  if (row_in) {
+  if (row_warp) {
+    // the chunk's unnormalised O (relative to m_run) out of tensor memory, 16 dims at a time, each
+    // group to the CTA that merges those dims
+    tc_fence_after();
+    const uint32_t o_lane = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)COL_O;   // this thread's lane, dim 0
     const uint32_t mine = smem_u32(recv + ((size_t)c * RR + row) * rs);
+#pragma unroll 1
+    for (int c0 = 0; c0 < DH; c0 += 16) {
+      uint32_t o[16];
+      if (have_o) {
+        tmem_ld16(o_lane + (uint32_t)c0, o);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      } else {
 #pragma unroll
-    for (int d = 0; d < ND; d += 4) {
-      const int gd = ND * half + d;
-      const int j = gd / wc;
-      const uint32_t a = mine + (uint32_t)(gd - j * wc) * 4;
-      st_cluster_v4(P.chunks > 1 ? peer_addr(a, (uint32_t)j) : a, acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
-    }
-    for (int j = 0; j < P.chunks; ++j) {
-      const uint32_t a = mine + (uint32_t)wc * 4;
+        for (int j = 0; j < 16; ++j) o[j] = 0u;
+      }
+      const int j = c0 / wc;
+      const uint32_t a = mine + (uint32_t)(c0 - j * wc) * 4;
       const uint32_t ra = P.chunks > 1 ? peer_addr(a, (uint32_t)j) : a;
-      if (half == 0) asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(ra), "f"(m_run), "f"(l_run) : "memory");
-      else asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra + 8), "f"(l_run) : "memory");
-      if (!DUP) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra + 8), "f"(0.f) : "memory");
+      if constexpr (DUP) {
+        // the query's two lanes hold the two parts of the pair's product: add them (both lanes get
+        // the sum) and let each lane store eight of the sixteen dims
+        float x[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const float lo8 = __uint_as_float(o[k]) + __shfl_xor_sync(0xffffffffu, __uint_as_float(o[k]), 16);
+          const float hi8 = __uint_as_float(o[8 + k]) + __shfl_xor_sync(0xffffffffu, __uint_as_float(o[8 + k]), 16);
+          x[k] = half ? hi8 : lo8;
+        }
+        if (row_in) {
+          st_cluster_v4(ra + (uint32_t)half * 32u, x[0], x[1], x[2], x[3]);
+          st_cluster_v4(ra + (uint32_t)half * 32u + 16u, x[4], x[5], x[6], x[7]);
+        }
+      } else if (row_in) {
+#pragma unroll
+        for (int k = 0; k < 16; k += 4)
+          st_cluster_v4(ra + (uint32_t)k * 4u, __uint_as_float(o[k]), __uint_as_float(o[k + 1]),
+                        __uint_as_float(o[k + 2]), __uint_as_float(o[k + 3]));
+      }
+    }
+    if (row_in) {
+#pragma unroll 1
+      for (int j = 0; j < P.chunks; ++j) {
+        const uint32_t a = mine + (uint32_t)wc * 4;
+        const uint32_t ra = P.chunks > 1 ? peer_addr(a, (uint32_t)j) : a;
+        if (half == 0) asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(ra), "f"(m_run), "f"(l_run) : "memory");
+        else asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra + 8), "f"(l_run) : "memory");
+        if (!DUP) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra + 8), "f"(0.f) : "memory");
+      }
     }
   }
   if (P.chunks > 1) cluster_sync_all(); else __syncthreads();
   if (row_in && !failed) {
     const int ncol = DUP ? wc / 2 : wc;                    // this thread's share of the CTA's dims
     const int col0 = DUP ? half * ncol : 0;
-    float mm = -INFINITY;
+    float mm = -INFINITY, l = 0.f;
+#pragma unroll 1
     for (int j = 0; j < P.chunks; ++j) mm = fmaxf(mm, recv[((size_t)j * RR + row) * rs + wc]);
-    float o[ND];
-#pragma unroll
-    for (int d = 0; d < ND; ++d) o[d] = 0.f;
-    float l = 0.f;
     if (mm != -INFINITY) {
+#pragma unroll 1
       for (int j = 0; j < P.chunks; ++j) {
-        const float *src = recv + ((size_t)j * RR + row) * rs;
-        const float4 ml = *reinterpret_cast<const float4 *>(src + wc);
-        if (ml.x == -INFINITY) continue;
-        const float w = exp2f(ml.x - mm);
-        l += w * (ml.y + ml.z);
-#pragma unroll
-        for (int d = 0; d < ND; d += 4) {
-          if (d < ncol) {
-            const float4 x = *reinterpret_cast<const float4 *>(src + col0 + d);
-            o[d] += w * x.x; o[d + 1] += w * x.y; o[d + 2] += w * x.z; o[d + 3] += w * x.w;
-          }
-        }
+        const float4 ml = *reinterpret_cast<const float4 *>(recv + ((size_t)j * RR + row) * rs + wc);
+        if (ml.x != -INFINITY) l += exp2f(ml.x - mm) * (ml.y + ml.z);
       }
     }
     const float inv = l > 0.f ? 1.f / l : 0.f;
     const size_t ob = (size_t)r_glob * H + h * DH + c * wc + col0;
-#pragma unroll
-    for (int d = 0; d < ND; d += 8) {
-      if (d < ncol) {
-        uint32_t hi[4], lo[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) split_pack(o[d + 2 * e] * inv, o[d + 2 * e + 1] * inv, hi[e], lo[e]);
-        *reinterpret_cast<uint4 *>(P.out + ob + d) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        if (P.out_lo != nullptr) *reinterpret_cast<uint4 *>(P.out_lo + ob + d) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+#pragma unroll 1
+    for (int d0 = 0; d0 < ncol; d0 += 8) {
+      float o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (mm != -INFINITY) {
+#pragma unroll 1
+        for (int j = 0; j < P.chunks; ++j) {               // in chunk order
+          const float *src = recv + ((size_t)j * RR + row) * rs;
+          const float mj = src[wc];
+          if (mj == -INFINITY) continue;
+          const float w = exp2f(mj - mm);
+          const float4 x0 = *reinterpret_cast<const float4 *>(src + col0 + d0);
+          const float4 x1 = *reinterpret_cast<const float4 *>(src + col0 + d0 + 4);
+          o[0] += w * x0.x; o[1] += w * x0.y; o[2] += w * x0.z; o[3] += w * x0.w;
+          o[4] += w * x1.x; o[5] += w * x1.y; o[6] += w * x1.z; o[7] += w * x1.w;
+        }
       }
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) split_pack(o[2 * e] * inv, o[2 * e + 1] * inv, hi[e], lo[e]);
+      *reinterpret_cast<uint4 *>(P.out + ob + d0) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      if (P.out_lo != nullptr) *reinterpret_cast<uint4 *>(P.out_lo + ob + d0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     }
   }
   if (warp == 5) {
@@ -525,11 +600,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
 
 int g_attn_tc_min_rows = 16;   // fewer query rows per sequence than this: the mma.sync kernel
 int g_attn_tc_chunks = 0;      // > 0: this many key chunks whatever the shape (A/B runs)
+int g_attn_tc_l2_ahead = 0;    // K/V tiles requested into L2 ahead of the ring
+int g_attn_tc_dry_pass = 1;
 
 }  // namespace
 
 void attn_tc_set_min_rows(int rows) { g_attn_tc_min_rows = rows; }
 void attn_tc_set_chunks(int chunks) { g_attn_tc_chunks = chunks; }
+void attn_tc_set_l2_ahead(int tiles) { g_attn_tc_l2_ahead = tiles < 0 ? 0 : tiles; }
+void attn_tc_set_dry_pass(int on) { g_attn_tc_dry_pass = on ? 1 : 0; }
 
 // Key chunks (= cluster size) per (sequence, head): the largest of 1, 2, 4, 8 that keeps the CTA
 // count within the SMs (one CTA per SM is resident; measured: a second, partly filled round and the
@@ -564,11 +643,13 @@ cudaError_t tree_attention_tc(Launch L, Operand q_pair, int q_rows_alloc, const 
   if (rows > 0x7fffffffLL) return cudaErrorInvalidValue;
   const int H = n_heads * DH;
   CUtensorMap tmQh, tmQl, tmK, tmV;
-  if (!tc_get_map(q_pair.hi, q_rows_alloc, H, 64, &tmQh) || !tc_get_map(q_pair.lo, q_rows_alloc, H, 64, &tmQl) ||
+  const int q_box = rows_per_seq <= 64 ? 16 : 64;      // rows per copy of the query operand
+  if (!tc_get_map(q_pair.hi, q_rows_alloc, H, q_box, &tmQh) || !tc_get_map(q_pair.lo, q_rows_alloc, H, q_box, &tmQl) ||
       !tc_get_map(k_cache, (int)rows, DH, TK, &tmK) || !tc_get_map(v_cache, (int)rows, DH, TK, &tmV))
     return cudaErrorInvalidValue;
   const int longest_first = (B > 1 && B <= 32 && (long long)chunks * B * n_heads > tc_num_sms()) ? 1 : 0;
-  AttnParams P{plan, (bf16 *)out.hi, (bf16 *)out.lo, rows_per_seq, n_heads, S_max, chunks, longest_first, status};
+  AttnParams P{plan, (bf16 *)out.hi, (bf16 *)out.lo, rows_per_seq, n_heads, S_max, chunks, longest_first,
+               g_attn_tc_l2_ahead, g_attn_tc_dry_pass, status};
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(chunks, n_heads * B);
   cfg.blockDim = dim3(THREADS);

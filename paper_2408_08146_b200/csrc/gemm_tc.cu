@@ -777,9 +777,13 @@ int tc_init_driver(char *err, size_t errlen) {
 
 void attn_tc_set_min_rows(int rows);
 void attn_tc_set_chunks(int chunks);
+void attn_tc_set_l2_ahead(int tiles);
+void attn_tc_set_dry_pass(int on);
 void tc_set_tuning(int key, int value) {
   if (key == 9) attn_tc_set_min_rows(value);
   if (key == 12) attn_tc_set_chunks(value);
+  if (key == 19) attn_tc_set_l2_ahead(value);
+  if (key == 20) attn_tc_set_dry_pass(value);
   if (key == 1) g_tune_stages = value;
   if (key == 10) g_tune_no_wave_split = value;
   if (key == 11) g_tune_no_wide = value;
