@@ -29,7 +29,9 @@ extern "C" {
  * MMAs; key 14 = weight tiles requested into L2 ahead of the ring in the 256-token form (default 0);
  * keys 15 (256-row weight tiles) and 16 (128-row tiles) = 1, 2 or 4: that many epilogue warps per
  * 32 accumulator lanes instead of the default; key 17 = 1: no CTA-pair GEMM kernel, 2: not up to 128
- * rows; key 18 = fewest rows for it (default 113). */
+ * rows; key 18 = fewest rows for it (default 113); key 19 = K/V tiles the
+ * tcgen05 attention requests into L2 ahead of its ring (default 0); key 20 = 0: no dry pass over its
+ * tile loop before the dependency wait. */
 void koala_set_tuning(int key, int value);
 
 /* Kernels launched by the library in this process so far (all contexts). */
