@@ -360,15 +360,24 @@ tree_attn_combine_kernel(const float *part, bf16 *__restrict__ out, bf16 *__rest
 
 }  // namespace
 
-// Key chunks per (sequence, head, row group): as many as keep the CTA count within the SMs, at
-// least one per 2048 keys of capacity, never finer than 256 keys of capacity per chunk.  One
-// chunk means one kernel (no partials, no combine).
+// Key chunks per (sequence, head, row group): as many as keep the CTA count within two CTAs per SM
+// (96 KB of shared memory each), at least one per 2048 keys of capacity, never finer than 128 keys of
+// capacity per chunk.  One chunk means one kernel (no partials, no combine).  (7B-shaped draft
+// iteration, 10 rows, context 1024: 1.965 / 1.905 / 1.858 / 1.845 / 1.839 ms with 1 / 2 / 4 / 6 / 8
+// chunks; 13B shape at batch 4, 160 sequence-head pairs: flat from 1 to 4, slower beyond.)
+int g_attn_mma_chunks = 0;     // > 0: this many key chunks whatever the shape (A/B runs)
+void attn_mma_set_chunks(int chunks) { g_attn_mma_chunks = chunks; }
 int attn_mma_chunks(int B, int n_heads, int rows_per_seq, int S_max, int num_sms) {
   const int rgs = (rows_per_seq + 15) / 16;
-  int c = num_sms / (rgs * B * n_heads);
+  if (g_attn_mma_chunks > 0) {
+    const int lim = S_max / 64 > 1 ? S_max / 64 : 1;
+    const int f = g_attn_mma_chunks > 16 ? 16 : g_attn_mma_chunks;
+    return f > lim ? lim : f;
+  }
+  int c = (2 * num_sms) / (rgs * B * n_heads);
   const int by_len = (S_max + 2047) / 2048;
   c = c < by_len ? by_len : c;
-  const int cap = S_max / 256 > 1 ? S_max / 256 : 1;
+  const int cap = S_max / 128 > 1 ? S_max / 128 : 1;
   c = c > cap ? cap : c;
   return c < 1 ? 1 : (c > 16 ? 16 : c);
 }

@@ -72,6 +72,7 @@ struct TcParams {
   int pf_ahead;       // weight tiles requested into L2 this many units ahead of the ring (0 = none)
   int early_w;        // how many of the first stages' weight tiles are requested before the dependency wait
   int l2_ahead;       // weight tiles prefetched into L2 beyond the ring before the dependency wait
+  int epi_dry;        // 1: the epilogue warps make a dry pass over their loop body (nothing stored) at kernel start
   int *status;
 };
 
@@ -298,7 +299,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     const int c_per = (((P.tt >> 4) + n_ch - 1) / n_ch) << 4;
     const int c_lo = min(((warp - 2) >> 2) * c_per, P.tt);
     const int c_hi = min(c_lo + c_per, P.tt);
-    pdl_wait();                          // the output buffer may still be read by the previous kernel
+    // A dry pass first: the loop body once with nothing stored and nothing waited for, while the
+    // first tiles stream - the epilogue's instructions are then already fetched when the first
+    // accumulator is complete.
+    bool dry = P.epi_dry != 0;
+    if (!dry) pdl_wait();                // the output buffer may still be read by the previous kernel
     bool ok = true;
     int seg = 0;
     unsigned u = u_lo;
@@ -307,13 +312,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
       unsigned seg_hi = (unsigned)(tile + 1) * KB;
       if (seg_hi > u_hi) seg_hi = u_hi;
       const int buf = seg % P.nbuf;
-      ok = mbar_wait(&acc_full[buf], (uint32_t)(seg / P.nbuf) & 1u);
-      if (!ok) break;
+      if (!dry) {
+        ok = mbar_wait(&acc_full[buf], (uint32_t)(seg / P.nbuf) & 1u);
+        if (!ok) break;
+      }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       int row0, col_off = 0, n_rows = P.n0;
       if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * bm; col_off = P.n0 + P.n1; n_rows = P.n2; }
       else if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * bm; col_off = P.n0; n_rows = P.n1; }
       else row0 = tile * bm;
+      if (dry) n_rows = 0;
       // which partial-sum slot: classic = the split index; stream-K = rank among the tile's contributors
       int slot = blockIdx.y;
       if (P.sk_ctas > 0)
@@ -359,6 +367,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
           }
         }
       }
+      }
+      if (dry) {                         // the same segment again, for real
+        dry = false;
+        pdl_wait();
+        continue;
       }
       // hand the accumulator buffer back to the MMA issuer
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -570,6 +583,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_const
     const int c_hi = min(c_lo + c_per, tt);
     const uint32_t acc_empty_even[2] = {cluster_addr_of(smem_u32(&acc_empty[0]), 0),
                                         cluster_addr_of(smem_u32(&acc_empty[1]), 0)};
+    bool dry = P.epi_dry != 0;           // a dry pass over the loop body first (nothing stored, nothing waited for)
     bool ok = true;
     int seg = 0;
     unsigned u = u_lo;
@@ -578,13 +592,16 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_const
       unsigned seg_hi = (unsigned)(tile + 1) * KB;
       if (seg_hi > u_hi) seg_hi = u_hi;
       const int buf = seg % P.nbuf;
-      ok = mbar_wait(&acc_full[buf], (uint32_t)(seg / P.nbuf) & 1u);
-      if (!ok) break;
+      if (!dry) {
+        ok = mbar_wait(&acc_full[buf], (uint32_t)(seg / P.nbuf) & 1u);
+        if (!ok) break;
+      }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       int row0, col_off = 0, n_rows = P.n0;
       if (tile >= P.tiles1) { row0 = (tile - P.tiles1) * PAIR_ROWS; col_off = P.n0 + P.n1; n_rows = P.n2; }
       else if (tile >= P.tiles0) { row0 = (tile - P.tiles0) * PAIR_ROWS; col_off = P.n0; n_rows = P.n1; }
       else row0 = tile * PAIR_ROWS;
+      if (dry) n_rows = 0;
       // partial-sum slot = rank of this cluster among the tile's contributors
       const int slot = (int)cid - (int)sk_owner((unsigned)tile * KB, (unsigned)P.sk_ctas, P.sk_units);
       for (int a = 0; a < 2; ++a) {
@@ -613,6 +630,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_const
             store16(vb, c0 + 16);
           }
         }
+      }
+      if (dry) {                         // the same segment again, for real
+        dry = false;
+        continue;
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -682,6 +703,7 @@ int g_tune_epi = 0;         // 1, 2: that many epilogue warps per lane quarter f
 int g_tune_epi_narrow = 0;  // 1, 2, 4: epilogue warps per lane quarter for 128-row weight tiles (default by token tile)
 int g_tune_no_pair2 = 0;    // 1 = no CTA-pair kernel; 2 = not for 65 to 128 tokens
 int g_tune_pair_min = 0;    // > 0: fewest rows for the CTA-pair kernel
+int g_tune_epi_dry = 1;
 int g_tune_pf = 0;           // > 0: weight tiles requested into L2 ahead of the ring in that mode
 int g_tune_no_wide = 0;      // 1 = 128 weight rows per CTA also for wide token tiles
 int g_tune_traffic_div = 8; // split <= K_in / (div * tokens)
@@ -779,6 +801,7 @@ void attn_tc_set_min_rows(int rows);
 void attn_tc_set_chunks(int chunks);
 void attn_tc_set_l2_ahead(int tiles);
 void attn_tc_set_dry_pass(int on);
+void attn_mma_set_chunks(int chunks);
 void tc_set_tuning(int key, int value) {
   if (key == 9) attn_tc_set_min_rows(value);
   if (key == 12) attn_tc_set_chunks(value);
@@ -793,6 +816,8 @@ void tc_set_tuning(int key, int value) {
   if (key == 16) g_tune_epi_narrow = value;
   if (key == 17) g_tune_no_pair2 = value;
   if (key == 18) g_tune_pair_min = value;
+  if (key == 21) g_tune_epi_dry = value;
+  if (key == 22) attn_mma_set_chunks(value);
   if (key == 2) g_tune_max_split = value;
   if (key == 3) g_tune_no_streamk = value;
   if (key == 5) g_tune_l2_ahead = value;
@@ -955,6 +980,7 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
       P.split = 1;
       P.split_stride = split_stride;
       P.status = status;
+      P.epi_dry = g_tune_epi_dry;
       CUtensorMap mw[3], mx, mxlo;
       for (int i = 0; i < 3; ++i) {
         const int j = i < m.n ? i : 0;
@@ -1059,6 +1085,7 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   P.split_stride = split_stride;
   P.status = status;
   P.nbuf = (sk && 2 * cols <= 256) ? 2 : 1;
+  P.epi_dry = g_tune_epi_dry;
   const int stage_bytes = (wide ? 2 : 1) * W_STAGE_BYTES + x_bytes;
   int stages = (g_smem_optin - 2048) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;

@@ -31,7 +31,8 @@ extern "C" {
  * 32 accumulator lanes instead of the default; key 17 = 1: no CTA-pair GEMM kernel, 2: not up to 128
  * rows; key 18 = fewest rows for it (default 113); key 19 = K/V tiles the
  * tcgen05 attention requests into L2 ahead of its ring (default 0); key 20 = 0: no dry pass over its
- * tile loop before the dependency wait. */
+ * tile loop before the dependency wait; key 21 = 0: no dry pass of the GEMM epilogue warps; key 22 =
+ * key chunks of the mma.sync attention kernel (0 = by rule). */
 void koala_set_tuning(int key, int value);
 
 /* Kernels launched by the library in this process so far (all contexts). */
