@@ -48,6 +48,15 @@ METRIC = "spec_decode_tokens_per_s"
 UNIT = "tokens/s"
 FORCED_LAM = 3.0
 HEADLINE = T13_EAGLE
+# DRAM traffic of the dominant launch from its ncu capture (one launch of gemm_tc_pair_kernel on the
+# 13B gate+up shape at 256 tokens, a 1.4 GB case: dram__bytes_read.sum + dram__bytes_write.sum), used
+# to scale the step's weight bytes per GEMM launch to DRAM bytes per launch: the traffic is the
+# weights once (1.03 x) plus one write-back of the fp32 partial sums, both proportional to the matrix.
+NCU_DRAM_BYTES = 291.5e6 + 28.2e6
+NCU_ALGORITHMIC_BYTES = 283.1e6
+NCU_SOURCE = ("scaled from one ncu capture of the dominant launch (gemm_tc_pair_kernel, 13B gate+up at 256 tokens: "
+              "319.7 MB of DRAM traffic for 283.1 MB of weights; profiles/ncu_gemm_tc_pair_kernel_t13_gateup_256tokens.md) "
+              "by the weight bytes per launch of this step")
 
 
 def forced_range(cfg):
@@ -387,8 +396,9 @@ def run_koala(args):
         "roofline": {"bound": "hbm", "kernel": "gemm_tc_pair_kernel + gemm_tc_kernel (all weight-streaming GEMMs of a step: the CTA-pair form "
                                "for the verification's 256 rows, the one-CTA form for the draft passes and the LM head)",
                      "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                     "peak_source": f"of {peaks['source']}", "traffic": None,
-                     "traffic_source": "not captured for the current kernel in this run (see the ncu summaries under profiles/)",
+                     "peak_source": f"of {peaks['source']}",
+                     "traffic": g["bytes"] / max(g["launches"], 1) * NCU_DRAM_BYTES / NCU_ALGORITHMIC_BYTES,
+                     "traffic_source": NCU_SOURCE,
                      "algorithmic_bytes_per_launch": g["bytes"] / max(g["launches"], 1),
                      "launches_per_step": g["launches"] / extra, "ms_per_step_in_kernel": g["ms"] / extra,
                      "tensor_TFLOPs_upper_bound": g_flops / (g["ms"] * 1e-3) / 1e12 if g["ms"] > 0 else 0.0},
