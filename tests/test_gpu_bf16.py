@@ -204,6 +204,14 @@ def test_t13_eagle_batch4_ragged():
     _teacher_forced_iteration(reduced(T13_EAGLE, 2))
 
 
+@pytest.mark.parametrize("B,N", [(2, 64), (2, 60), (4, 64), (1, 128)], ids=["2x64", "2x60", "4x64", "1x128"])
+def test_t7_shape_at_113_to_256_rows(B, N):
+    """The 7B shape at 120 to 256 verification rows: the GEMMs run as CTA pairs over 512-row weight
+    tiles; FFN 11008 = 21.5 tiles, so gate and up each end in a ragged tile and the second matrix
+    starts in the middle of one."""
+    _teacher_forced_iteration(reduced(T7_EAGLE, 2, K=1, B=B, N=N, S_max=640, prompt_len=384))
+
+
 @pytest.mark.parametrize("K", [2, 6])
 def test_t33_eagle_shape(K):
     """33B-shaped layers (hidden 6656, 52 heads, FFN 17920) with a deeper head; one target layer."""

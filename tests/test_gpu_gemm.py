@@ -68,3 +68,32 @@ def test_gemm_with_activation_pairs(shape, tc):
     err_pair = np.abs(y.cpu().numpy() - ref_full).max()
     err_bf16 = np.abs(hi.double().cpu().numpy() @ w.double().cpu().numpy().T - ref_full).max()
     assert err_pair < 0.05 * err_bf16 + 1e-5
+
+
+@pytest.mark.parametrize("shape", [(113, 1536, 1024), (128, 11008, 512), (129, 1024, 4096), (200, 700 * 16, 256),
+                                   (256, 5120, 5120), (256, 512, 13824)])
+def test_cta_pair_form_and_one_cta_form_agree(shape):
+    """113 to 256 rows as a pair of activations: the CTA-pair kernel (default) and the one-CTA kernel
+    (tuning key 17 = 1) both give the product of the pair's sum; ragged last tiles, one or many
+    K blocks, one or many tiles per cluster."""
+    from paper_2408_08146_b200 import binding
+    lib = binding.load_library()
+    M, N, K = shape
+    xf = normal_tensor(11, f"xf{M}.{N}.{K}", (M, K), 1.0, 0.0, torch.float32, "cuda:0")
+    w = normal_tensor(12, f"w{M}.{N}.{K}", (N, K), 0.02, 0.0, torch.bfloat16, "cuda:0")
+    hi = xf.to(torch.bfloat16)
+    lo = (xf - hi.float()).to(torch.bfloat16)
+    ref = (hi.double() + lo.double()).cpu().numpy() @ w.double().cpu().numpy().T
+    outs = []
+    try:
+        for off in (0, 1):
+            lib.koala_set_tuning(17, off)
+            status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+            y = koala_gemm_bf16(hi, w, True, 0, status, x_lo=lo)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            outs.append(y.cpu().numpy())
+            assert np.abs(outs[-1] - ref).max() <= 2e-5 * np.sqrt(K) + 1e-6
+    finally:
+        lib.koala_set_tuning(17, 0)
+    assert np.abs(outs[0] - outs[1]).max() <= 4e-5 * np.sqrt(K) + 1e-6
