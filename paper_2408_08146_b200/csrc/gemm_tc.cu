@@ -7,7 +7,8 @@
 // K = 16, both operands K-major in shared memory with the 128-byte swizzle that TMA writes.
 // The fp32 accumulator [128 x tokens] lives in tensor memory.  Warp 0 streams weight and
 // activation tiles with TMA through a ring of shared-memory stages (mbarrier full/empty pairs),
-// warp 1 issues the MMAs, warps 2..5 read the accumulator back (tcgen05.ld) and store it.
+// warp 1 issues the MMAs, four to sixteen epilogue warps read the accumulator back (tcgen05.ld,
+// one step ahead of the stores) and store it.
 // The weight stream does not depend on the previous kernel, so under programmatic dependent
 // launch the first stages are requested before waiting for the producer of X.
 // Activations may come as a pair hi + lo of bf16 matrices (lo = rounding residual of hi): the
@@ -18,7 +19,8 @@
 // accumulator columns, so a tile holds up to 256 tokens and the weights are passed over once.  With
 // 256 tokens a CTA takes 256 weight rows: four MMAs per K step share the activation tile and fill two
 // accumulators (all 512 tensor-memory columns); a stage is 32 KB of weights + 64 KB of activations,
-// two stages, one CTA per SM.
+// two stages, one CTA per SM.  From 113 rows up (as a pair) gemm_tc_pair_kernel takes over where it
+// applies: two CTAs of a cluster as one MMA unit, see there.
 // Split-K: grid.y CTAs share a weight tile and write separate partial outputs that the consumer
 // kernel sums in a fixed order (deterministic).
 // Every wait is bounded: on expiry the kernel records KOALA_E_TIMEOUT in *status, drains, frees
