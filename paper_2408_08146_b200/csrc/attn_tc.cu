@@ -140,7 +140,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
                     const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const AttnParams P) {
   constexpr int NC = DUP ? 32 : 64;      // keys of a tile per thread
-  constexpr int ND = DUP ? 64 : 128;     // output dims per thread
   constexpr int PB = DUP ? QSUB : P_BUF; // bytes of one P buffer
   constexpr int NST = DUP ? NKV + 1 : NKV;             // K/V stages
   constexpr int OKV = DUP ? OFF_KV - KV_STAGE : OFF_KV; // the ring starts where the second half of Q would be

@@ -42,8 +42,8 @@ namespace {
 constexpr int BM = 128;             // weight rows per CTA (MMA M)
 constexpr int BK = 64;              // K elements per stage: 128 bytes of bf16 = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int THREADS = 192;        // producer warp, MMA warp, four epilogue warps
-constexpr int THREADS_WIDE = 576;   // 256-row weight tiles: sixteen epilogue warps, four per 32 accumulator lanes
+constexpr int THREADS_WIDE = 576;   // most threads a launch uses: producer warp, MMA warp and sixteen epilogue
+                                    // warps (256-row weight tiles); 128-row tiles launch 192 or 320 threads
 constexpr int W_STAGE_BYTES = BM * BK * 2;
 constexpr int E_TIMEOUT = 6;
 constexpr int MAX_STAGES = 12;

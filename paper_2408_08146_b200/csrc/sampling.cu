@@ -137,7 +137,7 @@ accept_sampled_kernel(TreeBufs t, const float *verify_logits, const float *hid, 
   extern __shared__ float srow[];
   __shared__ Scratch sc;
   __shared__ int s_tok[128];
-  __shared__ int s_accept, s_len, s_bonus;
+  __shared__ int s_accept;
   pdl_launch_dependents();
   pdl_wait();
   const int b = blockIdx.x;
