@@ -494,7 +494,55 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
   constexpr int RR = DUP ? 64 : 128;     // rows per source chunk in the receive buffer
   float *recv = reinterpret_cast<float *>(sm + OKV);
   if (P.chunks > 1) cluster_sync_all();  // the receive buffer reuses the K/V ring: every CTA of the cluster is done with its tiles
-  if (row_warp) {
+  if (row_warp && P.chunks == 1) {
+    // one chunk: nothing to merge - O out of tensor memory 16 dims at a time, normalised and stored
+    tc_fence_after();
+    const uint32_t o_lane = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)COL_O;   // this thread's lane, dim 0
+    float l = l_run;
+    if (DUP) l += __shfl_xor_sync(0xffffffffu, l_run, 16);      // the query's other 32 keys of every tile
+    const float inv = (m_run != -INFINITY && l > 0.f) ? 1.f / l : 0.f;
+    const size_t ob = (size_t)r_glob * H + h * DH;
+#pragma unroll 1
+    for (int c0 = 0; c0 < DH; c0 += 16) {
+      uint32_t o[16];
+      if (have_o) {
+        tmem_ld16(o_lane + (uint32_t)c0, o);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) o[j] = 0u;
+      }
+      if constexpr (DUP) {
+        // the query's two lanes hold the two parts of the pair's product: add them; each lane stores eight dims
+        float x[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const float lo8 = __uint_as_float(o[k]) + __shfl_xor_sync(0xffffffffu, __uint_as_float(o[k]), 16);
+          const float hi8 = __uint_as_float(o[8 + k]) + __shfl_xor_sync(0xffffffffu, __uint_as_float(o[8 + k]), 16);
+          x[k] = (half ? hi8 : lo8) * inv;
+        }
+        if (row_in && !failed) {
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) split_pack(x[2 * e], x[2 * e + 1], hi[e], lo[e]);
+          const size_t at = ob + c0 + 8 * half;
+          *reinterpret_cast<uint4 *>(P.out + at) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          if (P.out_lo != nullptr) *reinterpret_cast<uint4 *>(P.out_lo + at) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+      } else if (row_in && !failed) {
+#pragma unroll
+        for (int g8 = 0; g8 < 2; ++g8) {
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            split_pack(__uint_as_float(o[8 * g8 + 2 * e]) * inv, __uint_as_float(o[8 * g8 + 2 * e + 1]) * inv, hi[e], lo[e]);
+          const size_t at = ob + c0 + 8 * g8;
+          *reinterpret_cast<uint4 *>(P.out + at) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          if (P.out_lo != nullptr) *reinterpret_cast<uint4 *>(P.out_lo + at) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+      }
+    }
+  } else if (row_warp) {
     // the chunk's unnormalised O (relative to m_run) out of tensor memory, 16 dims at a time, each
     // group to the CTA that merges those dims
     tc_fence_after();
@@ -546,7 +594,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
     }
   }
   if (P.chunks > 1) cluster_sync_all(); else __syncthreads();
-  if (row_in && !failed) {
+  if (row_in && !failed && P.chunks > 1) {
     const int ncol = DUP ? wc / 2 : wc;                    // this thread's share of the CTA's dims
     const int col0 = DUP ? half * ncol : 0;
     float mm = -INFINITY, l = 0.f;
