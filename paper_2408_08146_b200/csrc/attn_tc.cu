@@ -365,8 +365,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQh, const __grid_const
       if (t == 0) {
         read_plan();
         T_run = T;
+        r_glob = b * P.rows_per_seq + (row_in ? row : 0);    // also needed by a chunk without tiles: it still merges and stores its dims
         if (T == 0) break;
-        r_glob = b * P.rows_per_seq + (row_in ? row : 0);
         ok_row = row_in && P.plan.slot[r_glob] >= 0;
         mk0 = ok_row ? P.plan.mask[(size_t)r_glob * 2] : 0ull;
         mk1 = ok_row ? P.plan.mask[(size_t)r_glob * 2 + 1] : 0ull;

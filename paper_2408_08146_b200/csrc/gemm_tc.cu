@@ -43,7 +43,7 @@ constexpr int BM = 128;             // weight rows per CTA (MMA M)
 constexpr int BK = 64;              // K elements per stage: 128 bytes of bf16 = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int THREADS_WIDE = 576;   // most threads a launch uses: producer warp, MMA warp and sixteen epilogue
-                                    // warps (256-row weight tiles); 128-row tiles launch 192 or 320 threads
+                                    // warps (256-row weight tiles); 128-row tiles launch 320 threads
 constexpr int W_STAGE_BYTES = BM * BK * 2;
 constexpr int E_TIMEOUT = 6;
 constexpr int MAX_STAGES = 12;
@@ -1117,10 +1117,10 @@ cudaError_t gemm_tc(Launch L, Operand X, int x_rows_alloc, GemmMats m, int K_in,
   }
   // Epilogue warps per 32 accumulator lanes.  256-row tiles keep one accumulator set, so the MMAs
   // of a CTA's next tile wait for the epilogue: sixteen warps (13B-shaped verification of 256 rows:
-  // 18.3 ms with four, 16.8 with eight, 16.3 with sixteen).  128-row tiles: eight warps up to 48
-  // tokens (measured 2-3 % faster per verification and per draft pass, 8 to 48 tokens), four beyond
-  // (64 and 128 tokens measured 1-2 % slower with eight).
-  int groups = wide ? 4 : (tt <= 48 ? 2 : 1);
+  // 18.3 ms with four, 16.8 with eight, 16.3 with sixteen).  128-row tiles: eight warps (per 7B
+  // verification, against four: 16 to 48 rows 2-3 % faster, 60 and 64 rows 1 %, 100 rows 0.8 %,
+  // 80 rows 0.5 % slower; the draft passes 2 % faster).
+  int groups = wide ? 4 : 2;
   const int forced = wide ? g_tune_epi : g_tune_epi_narrow;
   if (forced == 1 || forced == 2 || forced == 4) groups = forced;
   return launch_k(gemm_tc_kernel, grid, dim3(64 + 128 * groups), smem, L.st, L.pdl, mw[0], mw[1], mw[2], mx, mxlo, P);

@@ -121,7 +121,9 @@ def test_long_context_many_key_tiles_and_chunks(context):
     (20, 1, 32, 300, 512),       # fewer than 32 rows: one row group, duplicated
     (40, 8, 32, 200, 512),       # more CTAs than SMs: a single chunk, no cluster
     (60, 1, 8, 3000, 4096),      # few heads: 8 key chunks per head
-    (33, 1, 32, 64, 256),        # context shorter than a chunk's share: empty chunks
+    (33, 1, 32, 64, 256),        # a short context: one tile per chunk
+    (33, 1, 32, 20, 1024),       # one key tile, four key chunks: three CTAs of a cluster have no tile and still merge and store their dims
+    (60, 1, 8, 10, 4096),        # two key tiles, eight key chunks
 ])
 def test_tensor_core_attention_shapes(N, B, n_heads, context, S_max):
     """One bf16 layer with head_dim 128 at row counts, batch sizes and chunk counts that select
@@ -271,3 +273,32 @@ def test_position_wise_acceptance_counters_match_the_oracle():
     assert eng.koala_accept_stats(cfg.N) == ([0] * cfg.N, [0] * cfg.N)
     assert eng.device_status() == 0
     eng.close()
+
+
+def test_whole_iterations_repeat_bit_for_bit():
+    """Two engines on the same weights, prompts ingested in chunks (the first chunks have fewer key
+    tiles than key chunks), several forced iterations: trees, target tokens and accepted tokens must
+    be identical."""
+    from workloads import T7_EAGLE, reduced
+    from workloads.generate import WeightStore
+    from paper_2408_08146_b200 import Koala
+    cfg = reduced(T7_EAGLE, 2, K=1, S_max=768, prompt_len=300)
+    store = WeightStore(cfg, DEV)
+    forced = torch.tensor([[3], [1], [5], [2]], dtype=torch.int32, device=DEV)
+    runs = []
+    for _ in range(2):
+        eng = Koala(cfg, store.tensors)
+        eng.prefill(prompts(cfg), 64)
+        rec = [eng.buffers()["root_tok"].cpu().numpy().copy()]
+        for i in range(forced.shape[0]):
+            toks, lens = eng.step(forced[i])
+            torch.cuda.synchronize()
+            b = eng.buffers()
+            n = int(b["tree_n"][0].item())
+            rec += [lens.cpu().numpy().copy(), toks[0, :int(lens[0].item())].cpu().numpy().copy(),
+                    b["tree_tok"][0, :n].cpu().numpy().copy(), b["verify_tgt"][:n].cpu().numpy().copy()]
+        assert eng.device_status() == 0
+        eng.close()
+        runs.append(rec)
+    for a, c in zip(*runs):
+        assert np.array_equal(a, c)
